@@ -1,0 +1,310 @@
+"""Pins for the oracle's scalar preparation, the AdamW step of Algorithm 2 and EDQ (Eq. 2-3).
+
+Fixed by: Table 1 (beta2 expansions), the closed forms of Section 3.2 ("in the
+absence of imprecision EDQ is the norm of the update"), Section 4.2 (second
+moment grows monotonically when beta2 rounds to 1), exact rational brute force
+on single parameters, and agreement with AdamW in double within what a
+length-2 bfloat16 expansion can hold.
+"""
+from pathlib import Path
+
+import numpy as np
+import pytest
+
+import oracle
+from conftest import bf16_window, bits_to_f64, ulp_f64
+import exact_rational as R
+from paper_2405_03637_b200 import workloads as W
+
+GOLDEN = Path(__file__).resolve().parent / "golden"
+HYP = dict(lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
+
+
+def _records(name):
+    out = {}
+    for line in (GOLDEN / name).read_text().splitlines():
+        if line.startswith("#") or not line.strip():
+            continue
+        parts = [p.strip() for p in line.split("|")]
+        out[parts[0]] = parts[1]
+    return out
+
+
+def _state(theta_bits, strategy):
+    th = np.array(theta_bits, dtype=np.uint16)
+    z = lambda: np.zeros_like(th)
+    return dict(x_hi=th, x_lo=z() if strategy >= 1 else None, m=z(), v_hi=z(), v_lo=z() if strategy == 2 else None)
+
+
+def _step(st, g, t, strategy, hyp=HYP, **kw):
+    return oracle.adamw_step(st["x_hi"], st["x_lo"], st["m"], st["v_hi"], st["v_lo"], g, step=t,
+                             strategy=strategy, **hyp, **kw)
+
+
+# ------------------------------------------------------------------ scalars ---
+
+def test_beta2_expansions_match_table_1():
+    rec = _records("paper_values.txt")
+    for b2 in (0.999, 0.99, 0.95):
+        hi_txt, lo_txt = rec[f"beta2_expansion_{b2}"].split()
+        sc = oracle.derive_scalars(1e-4, 0.9, b2, 1e-8, 0.1, 1)
+        hi, lo = oracle.widen(sc["b2h"]), oracle.widen(sc["b2l"])
+        if b2 == 0.99:
+            hi_txt = "0.9883"   # the table's 0.9893 is a misprint: 0.9893 + 0.0017 != 0.99
+        digits = len(hi_txt.split(".")[1]) if "." in hi_txt else 0
+        assert round(hi, digits) == float(hi_txt)
+        assert round(lo, 4) == float(lo_txt) or round(lo, 3) == float(lo_txt)
+        # the expansion represents beta2 to about 16 bits, and the first component alone does not
+        assert abs(hi + lo - b2) < 2.0 ** -16
+        assert abs(hi - b2) > 2.0 ** -11
+        assert abs(lo) <= float(ulp_f64(np.array([sc["b2h"]], np.uint16))[0]) / 2
+    sc = oracle.derive_scalars(1e-4, 0.9, 0.999, 1e-8, 0.1, 1)
+    assert (sc["b2h"], oracle.widen(sc["b2l"])) == (0x3F80, -0.00099945068359375)
+
+
+def test_scalars_against_exact_rationals():
+    rec = _records("worked_values.txt")
+    for t in (1, 2, 3, 10, 100, 1000):
+        want = dict(kv.split("=") for kv in rec[f"scalars t={t}"].split())
+        got = oracle.derive_scalars(1e-4, 0.9, 0.999, 1e-8, 0.1, t)
+        assert {k: f"{v:04X}" for k, v in got.items()} == want
+    for b2 in ("0.999", "0.99", "0.98", "0.95"):
+        got = oracle.derive_scalars(1e-4, 0.9, float(b2), 1e-8, 0.1, 1)
+        assert f"{got['b2h']:04X} {got['b2l']:04X}" == rec[f"beta2 {b2}"]
+    # bias corrections computed in double before the cast (Appendix D): they approach 1 from below, monotonically
+    prev = 0.0
+    for t in range(1, 3000):
+        bc2 = oracle.widen(oracle.derive_scalars(1e-4, 0.9, 0.999, 1e-8, 0.1, t)["bc2"])
+        assert prev <= bc2 <= 1.0
+        assert abs(bc2 - (1 - 0.999 ** t)) <= 2.0 ** -8 * bc2
+        prev = bc2
+
+
+def test_primitive_worked_values():
+    rec = _records("worked_values.txt")
+    a = lambda *xs: [np.array([int(x, 16)], np.uint16) for x in xs]
+    fmt = lambda pair: f"{int(pair[0][0]):04X} {int(pair[1][0]):04X}"
+    for key, want in rec.items():
+        name, *args = key.split()
+        if name == "fast_two_sum":
+            assert fmt(oracle.fast_two_sum(*a(*args))) == want
+            assert fmt(oracle.two_sum(*a(*reversed(args)))) == want
+        elif name == "two_prod":
+            assert fmt(oracle.two_prod(*a(*args))) == want
+        elif name == "mul":
+            assert fmt(oracle.mul(*a(*args))) == want
+        elif name == "scaling":
+            assert fmt(oracle.scaling(*a(*args))) == want
+
+
+# -------------------------------------------------------------- step traces ---
+
+@pytest.mark.parametrize("strategy", [0, 1, 2])
+def test_single_parameter_trace(strategy):
+    rec = _records("worked_values.txt")
+    st = _state([0x3CA4], strategy)
+    g = np.array([0x3A83], np.uint16)
+    for t in range(1, 6):
+        _, d = _step(st, g, t, strategy, want_delta=True)
+        want = dict(kv.split("=") for kv in rec[f"trace strategy={strategy} t={t}"].split())
+        got = dict(th=st["x_hi"], dth=st["x_lo"], m=st["m"], v=st["v_hi"], dv=st["v_lo"], delta=d)
+        for k, arr in got.items():
+            assert f"{(int(arr[0]) if arr is not None else 0):04X}" == want[k], (t, k)
+
+
+@pytest.mark.parametrize("strategy", [1, 2])
+def test_second_trace_eps_inside_and_sign_changes(strategy):
+    rec = _records("worked_values.txt")
+    hyp = dict(HYP, beta2=0.95, lr=3e-3)
+    st = _state([0xBF13], strategy)
+    for t, g in enumerate([0x3B21, 0xBA05, 0x3C7F, 0x0000, 0xB9C4, 0x3B21], start=1):
+        _, d = _step(st, np.array([g], np.uint16), t, strategy, hyp=hyp, want_delta=True,
+                     flags=oracle.FLAG_EPS_INSIDE_SQRT)
+        want = dict(kv.split("=") for kv in rec[f"trace2 strategy={strategy} t={t} g={g:04X}"].split())
+        got = dict(th=st["x_hi"], dth=st["x_lo"], m=st["m"], v=st["v_hi"], dv=st["v_lo"], delta=d)
+        for k, arr in got.items():
+            assert f"{(int(arr[0]) if arr is not None else 0):04X}" == want[k], (t, k)
+
+
+def test_random_single_parameters_against_exact_rationals():
+    rng = np.random.default_rng(8)
+    thetas = rng.choice(bf16_window(-9, 1), 40)
+    hyp = dict(lr=2e-3, beta1=0.9, beta2=0.98, eps=1e-8, weight_decay=0.01)
+    for strategy in (0, 1, 2):
+        for eps_inside in (False, True):
+            st = _state(thetas.copy(), strategy)
+            ref = [(int(b), 0, 0, 0, 0) for b in thetas]
+            for t in range(1, 7):
+                g = rng.choice(bf16_window(-14, -6), thetas.size)
+                _, d = _step(st, g, t, strategy, hyp=hyp, want_delta=True,
+                             flags=oracle.FLAG_EPS_INSIDE_SQRT if eps_inside else 0)
+                sc = R.scalars("2e-3", "0.9", "0.98", "1e-8", "0.01", t)
+                for i in range(thetas.size):
+                    *ref_i, delta = R.adamw_element(*ref[i], int(g[i]), sc, strategy, eps_inside)
+                    ref[i] = tuple(ref_i)
+                    got = (int(st["x_hi"][i]), int(st["x_lo"][i]) if strategy else 0, int(st["m"][i]),
+                           int(st["v_hi"][i]), int(st["v_lo"][i]) if strategy == 2 else 0)
+                    same = all(a == b or ((a | b) & 0x7FFF) == 0 for a, b in zip(got, ref[i]))
+                    assert same and int(d[i]) == delta, (strategy, eps_inside, t, i)
+                    ref[i] = got       # keep zero signs of the oracle so later steps see identical inputs
+
+
+# --------------------------------------------------------------- closed forms ---
+
+def test_edq_equals_update_norm_when_grow_is_exact():
+    # Section 3.2: with no imprecision EDQ is the norm of the intended update.  With |theta| >= |delta| and
+    # an empty second component, Grow is error-free, so strategies B and C apply the update exactly.
+    n = 1 << 16
+    th = W.bits(W.flat_weights(n, 0))
+    th = np.where(np.abs(bits_to_f64(th)) < 1e-3, np.uint16(0x3CA4), th)
+    g = W.bits(W.flat_grads(n, 0, 1))
+    for strategy in (1, 2):
+        st = _state(th.copy(), strategy)
+        sums, d = _step(st, g, 1, strategy, want_delta=True)
+        norm = float(np.sqrt(np.sum(bits_to_f64(d) ** 2)))
+        assert sums["edq"] == pytest.approx(norm, rel=1e-12)
+        assert sums["lost"] == 0
+        applied = (bits_to_f64(st["x_hi"]) + bits_to_f64(st["x_lo"])) - bits_to_f64(th)
+        assert np.array_equal(applied, bits_to_f64(d))
+    # plain bfloat16 applies a different vector (lost and over-moved elements): EDQ departs from the norm,
+    # and Cauchy-Schwarz still bounds it by the norm of the effective update
+    st = _state(th.copy(), 0)
+    sums, d = _step(st, g, 1, 0, want_delta=True)
+    eff = bits_to_f64(st["x_hi"]) - bits_to_f64(th)
+    norm = float(np.sqrt(np.sum(bits_to_f64(d) ** 2)))
+    assert sums["edq"] > 0 and abs(sums["edq"] - norm) > 1e-3 * norm
+    assert abs(sums["edq"]) <= float(np.sqrt(np.sum(eff ** 2))) * (1 + 1e-12)
+    assert sums["lost"] == int(np.sum((bits_to_f64(d) != 0) & (eff == 0)))
+    assert sums["lost"] > 0
+
+
+def test_plain_bf16_loses_every_small_update_and_collage_keeps_it():
+    # all |delta| far below ulp(theta)/2: option A leaves theta unchanged (EDQ = 0, Def. 3.2), B keeps it in dtheta
+    n = 4096
+    th = np.full(n, oracle.round_to_bf16(200.0), np.uint16)
+    g = W.bits(W.flat_grads(n, 3, 1))
+    stA, stB = _state(th.copy(), 0), _state(th.copy(), 1)
+    hyp = dict(HYP, weight_decay=0.0)
+    sA, dA = _step(stA, g, 1, 0, hyp=hyp, want_delta=True)
+    sB, dB = _step(stB, g, 1, 1, hyp=hyp, want_delta=True)
+    nz = bits_to_f64(dA) != 0
+    assert nz.sum() > n * 0.9 and np.all(np.abs(bits_to_f64(dA)) < 0.5)
+    assert np.array_equal(stA["x_hi"], th) and sA["edq"] == 0.0 and sA["lost"] == int(nz.sum())
+    assert np.array_equal(stB["x_hi"], th) and np.array_equal(stB["x_lo"], dB)
+    assert sB["edq"] == pytest.approx(float(np.sqrt(np.sum(bits_to_f64(dB) ** 2))), rel=1e-12)
+    assert sB["lost"] == 0
+
+
+def test_edq_single_parameter_closed_form_and_zero_norm():
+    st = _state([0x3CA4], 0)
+    sums, d = _step(st, np.array([0x3A83], np.uint16), 1, 0, want_delta=True)
+    eff = bits_to_f64(st["x_hi"])[0] - bits_to_f64(np.array([0x3CA4], np.uint16))[0]
+    assert sums["edq"] == pytest.approx(np.sign(bits_to_f64(d)[0]) * eff, rel=1e-15)
+    # zero gradient and zero weight decay: no update, EDQ defined as 0
+    st = _state([0x3CA4], 1)
+    sums, d = _step(st, np.array([0], np.uint16), 1, 1, hyp=dict(HYP, weight_decay=0.0), want_delta=True)
+    assert (bits_to_f64(d)[0], sums["sumsq"], sums["edq"]) == (0.0, 0.0, 0.0)
+    # the stand-alone EDQ routine agrees with the fused one
+    n = 10_000
+    th = W.bits(W.flat_weights(n, 5)); g = W.bits(W.flat_grads(n, 5, 1))
+    st = _state(th.copy(), 2)
+    sums, d = _step(st, g, 1, 2, want_delta=True)
+    alone = oracle.edq(th, np.zeros_like(th), st["x_hi"], st["x_lo"], d)
+    assert alone == sums
+    # threads only change the association of the two sums
+    st2 = _state(th.copy(), 2)
+    sums2, _ = _step(st2, g, 1, 2, threads=3)
+    assert sums2["edq"] == pytest.approx(sums["edq"], rel=1e-13) and sums2["lost"] == sums["lost"]
+    assert all(np.array_equal(st[k], st2[k]) for k in st)
+
+
+def test_second_moment_monotone_without_expansion_and_tracks_with_it():
+    # Section 4.2: beta2 = 0.999 rounds to 1.0 in bfloat16, so under A/B v can only grow; under C it follows the EMA
+    n = 2048
+    th = W.bits(W.flat_weights(n, 6))
+    stB, stC = _state(th.copy(), 1), _state(th.copy(), 2)
+    v64 = np.zeros(n)
+    for t in range(1, 401):
+        g = W.bits(W.flat_grads(n, 6, t))
+        prev = bits_to_f64(stB["v_hi"]).copy()
+        _step(stB, g, t, 1)
+        _step(stC, g, t, 2)
+        assert np.all(bits_to_f64(stB["v_hi"]) >= prev)
+        v64 = 0.999 * v64 + 0.001 * bits_to_f64(g) ** 2
+    vC = bits_to_f64(stC["v_hi"]) + bits_to_f64(stC["v_lo"])
+    vB = bits_to_f64(stB["v_hi"])
+    relC = np.abs(vC - v64) / v64
+    assert np.median(relC) < 0.01 and relC.max() < 0.05
+    # the monotone sum overshoots the average it should be (sum of increments vs. decayed average)
+    assert np.median(vB / v64) > 1.1
+    assert np.all(np.abs(bits_to_f64(stC["v_lo"])) <= ulp_f64(stC["v_hi"]) / 2)
+
+
+# ------------------------------------------------------ against AdamW in double ---
+
+def test_collage_accumulates_its_own_updates_exactly_where_plain_bf16_does_not():
+    # shadow test: sum in double the bfloat16 updates each strategy actually produced; a length-2 expansion
+    # tracks that sum to within the roundings of its second component, a single bfloat16 does not
+    n = 8192
+    th0 = W.bits(W.stress_weights(n, 2))
+    hyp = dict(W.HYPERS_STRESS)
+    err = {}
+    for strategy in (0, 2):
+        st = _state(th0.copy(), strategy)
+        shadow = bits_to_f64(th0).copy()
+        bound = np.zeros(n)
+        for t in range(1, 61):
+            g = W.bits(W.stress_grads(n, 2, t))
+            _, d = _step(st, g, t, strategy, hyp=hyp, want_delta=True)
+            shadow += bits_to_f64(d)
+            if strategy:
+                bound += ulp_f64(st["x_lo"]) / 2 + 2.0 ** -140
+        held = bits_to_f64(st["x_hi"]) + (bits_to_f64(st["x_lo"]) if strategy else 0.0)
+        err[strategy] = np.abs(held - shadow)
+        if strategy:
+            assert np.all(err[strategy] <= bound)
+    assert err[2].sum() < 0.02 * err[0].sum()
+
+
+def test_step_agrees_with_fp64_adamw_within_mcf_precision():
+    n = 1 << 14
+    th0 = W.bits(W.flat_weights(n, 0))
+    T = 50
+    hyp = dict(HYP, beta2=0.95)
+    th64 = bits_to_f64(th0).copy(); m64 = np.zeros(n); v64 = np.zeros(n)
+    moved = np.zeros(n)
+    states = {s: _state(th0.copy(), s) for s in (0, 1, 2)}
+    for t in range(1, T + 1):
+        g = W.bits(W.flat_grads(n, 0, t))
+        d64 = oracle.adamw_fp64(th64, m64, v64, bits_to_f64(g), step=t, want_delta=True, **hyp)
+        moved += np.abs(d64)
+        for s, st in states.items():
+            _step(st, g, t, s, hyp=hyp)
+    dist = {}
+    for s, st in states.items():
+        held = bits_to_f64(st["x_hi"]) + (bits_to_f64(st["x_lo"]) if s else 0.0)
+        dist[s] = np.abs(held - th64)
+    # each bfloat16 update carries ~2^-8 relative rounding per operation over a chain of 8; 5% of the path
+    # length bounds their accumulation, plus the resolution of the expansion itself
+    for s in (1, 2):
+        assert np.all(dist[s] <= 0.05 * moved + T * 2.0 ** -16 * np.abs(th64))
+    # and Collage sits far closer to the fp64 trajectory than plain bfloat16
+    assert dist[1].sum() < 0.25 * dist[0].sum()
+    assert dist[2].sum() < 0.25 * dist[0].sum()
+    # the fp64 routine itself against a two-line numpy restatement of AdamW at t = 1 (m = v = 0)
+    g = bits_to_f64(W.bits(W.flat_grads(n, 0, 1)))
+    th = bits_to_f64(th0).copy(); m = np.zeros(n); v = np.zeros(n)
+    oracle.adamw_fp64(th, m, v, g, step=1, **HYP)
+    want = bits_to_f64(th0) - 1e-4 * (g / (np.abs(g) + 1e-8) + 0.1 * bits_to_f64(th0))
+    assert np.allclose(th, want, rtol=1e-12, atol=0)
+
+
+def test_bytes_per_parameter_accounting():
+    rec = _records("paper_values.txt")
+    want = [int(x) for x in rec["bytes_per_parameter_A_B_C_D"].split()]
+    n = 64
+    sizes = []
+    for s in (0, 1, 2):
+        st = W.fresh_state(W.flat_weights(n, 0), s)
+        sizes.append((sum(t.numel() * t.element_size() for t in st.arrays()) + n * 2) // n)   # + gradient
+    assert sizes == want[:3]
