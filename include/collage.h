@@ -1,0 +1,171 @@
+/*
+ * collage.h -- C ABI of the B200 (sm_100a) Collage bf16 multi-component-float AdamW library.
+ *
+ * The library implements the optimizer step of "Collage: Light-Weight Low-Precision Strategy
+ * for LLM Training" (Algorithm 2) for the paper's precision options A (plain bfloat16),
+ * B (Collage-light: theta held as a bfloat16 pair) and C (Collage-plus: theta and the second
+ * moment held as pairs, beta2 as a pair), the error-free transforms it is built from
+ * (Theorem 4.1, Algorithm 1, Appendix C), and the effective-descent-quality metric (Eq. 2-3).
+ *
+ * Arithmetic model (Section 3.1): every operator written in the paper takes bfloat16 operands
+ * and rounds its exact result once, to nearest-even, to bfloat16.  Scalars are evaluated in
+ * double on the host and cast to bfloat16 last (Section 4.2, Appendix D).
+ *
+ * Conventions for every entry point unless it says otherwise:
+ *   - tensor pointers are DEVICE pointers to bfloat16 bit patterns (uint16_t), owned by the
+ *     caller, on the current CUDA device; hyper-parameter structs, tensor lists and scalar
+ *     outputs named "host" are HOST pointers;
+ *   - state tensors are updated in place; `grad` is read only;
+ *   - calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default
+ *     stream); the library never synchronises the device and never allocates on the step path;
+ *   - errors are detected on the host BEFORE anything is launched and reported as a status
+ *     code; nothing is thrown across the boundary; there is no CPU fallback: a device that is
+ *     not compute capability 10.x yields COLLAGE_ERR_ARCH;
+ *   - pointers need not be 16-byte aligned and lengths need not be multiples of 8 (such
+ *     tensors take a slower element-wise path with identical results);
+ *   - n == 0 is a successful no-op;
+ *   - NaN/Inf in tensor data is not an error: it propagates per IEEE 754.
+ */
+#ifndef COLLAGE_H_
+#define COLLAGE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    COLLAGE_OK = 0,
+    COLLAGE_ERR_NULL = 1,       /* a required pointer is NULL                                   */
+    COLLAGE_ERR_ARG = 2,        /* step == 0, unknown strategy/op, hyper-parameter out of range */
+    COLLAGE_ERR_ALIAS = 3,      /* two tensors of one call overlap                              */
+    COLLAGE_ERR_ARCH = 4,       /* current device is not sm_100                                 */
+    COLLAGE_ERR_CUDA = 5,       /* a CUDA runtime call or launch failed                         */
+    COLLAGE_ERR_WORKSPACE = 6   /* workspace missing or smaller than collage_workspace_bytes()  */
+} collage_status_t;
+
+/* Precision options of Table 2. */
+typedef enum {
+    COLLAGE_BF16 = 0,   /* A: theta, m, v single bfloat16                    ( 8 B/param with grad) */
+    COLLAGE_LIGHT = 1,  /* B: (theta, dtheta) pair                           (10 B/param)           */
+    COLLAGE_PLUS = 2    /* C: (theta, dtheta), (v, dv) pairs, beta2 as pair  (12 B/param)           */
+} collage_strategy_t;
+
+/* Algorithm 2 line 12 prints epsilon under the root; AdamW has it outside.  Default: outside. */
+#define COLLAGE_FLAG_EPS_INSIDE_SQRT 1u
+
+/* Hyper-parameters of one step (Algorithm 2 line 1).  HOST struct.
+ * Valid ranges: lr, eps, weight_decay >= 0 and finite; 0 <= beta1, beta2 < 1. */
+typedef struct collage_hyper {
+    double lr, beta1, beta2, eps, weight_decay;
+    uint32_t flags;          /* COLLAGE_FLAG_*                                                   */
+    void* edq_out;           /* DEVICE collage_edq_t*, or NULL to skip the EDQ reduction          */
+    void* workspace;         /* DEVICE scratch, >= collage_workspace_bytes(); needed iff edq_out  */
+    size_t workspace_bytes;
+} collage_hyper_t;
+
+/* Result of the EDQ reduction (Eq. 3), written on the device by the call's last kernel.
+ *   dot   = sum_i delta_i * eff_i        eff = (theta'+dtheta') - (theta+dtheta)   (Eq. 2)
+ *   sumsq = sum_i delta_i^2              delta = the bfloat16 update of Algorithm 2 line 12
+ *   edq   = dot / sqrt(sumsq), 0 if sumsq == 0
+ *   lost  = #{i : delta_i != 0 and no component of the stored parameter changed} (Def. 3.2)
+ * Products and 8-element partial sums are formed in float, everything above in double, in a
+ * fixed order: the result is reproducible for a given launch geometry. */
+typedef struct collage_edq {
+    double dot, sumsq, edq;
+    uint64_t n;
+    uint64_t lost;
+} collage_edq_t;
+
+/* One parameter tensor of a multi-tensor plan.  x_lo may be NULL for a plan used only with
+ * COLLAGE_BF16; v_lo may be NULL unless the plan is used with COLLAGE_PLUS. */
+typedef struct collage_tensor {
+    void* x_hi;        /* theta          */
+    void* x_lo;        /* delta-theta    */
+    void* m;           /* first moment   */
+    void* v_hi;        /* second moment  */
+    void* v_lo;        /* delta-v        */
+    const void* grad;
+    uint64_t n;        /* elements       */
+} collage_tensor_t;
+
+typedef struct collage_plan collage_plan_t;   /* opaque; owns a small device table */
+
+const char* collage_status_string(collage_status_t status);
+
+/* Scalar preparation (Algorithm 2 line 1; Table 1; Appendix D "Scalar and Bias Correction").
+ * HOST only, no CUDA call.  out_bf16[11] receives, as bfloat16 bit patterns,
+ *   [0] RN(beta1) [1] RN(1-beta1) [2] RN(beta2) [3] RN(1-beta2)
+ *   [4] beta2_hi = RN(beta2) [5] beta2_lo = RN(beta2 - beta2_hi)
+ *   [6] RN(1-beta1^step) [7] RN(1-beta2^step) [8] RN(lr) [9] RN(weight_decay) [10] RN(eps)
+ * every expression evaluated in double before the one rounding.
+ * Errors: NULL -> ERR_NULL; step == 0 or hyper out of range -> ERR_ARG. */
+collage_status_t collage_derive_scalars(const collage_hyper_t* hyper, uint64_t step, uint16_t out_bf16[11]);
+
+/* Bytes of device scratch the EDQ reduction needs (independent of n; a few tens of KiB). */
+size_t collage_workspace_bytes(uint64_t n_total);
+
+/* One AdamW step over one flat tensor (Algorithm 2 lines 8-13, all n parameters, step t >= 1).
+ *   x_hi, m, v_hi, grad : required.   x_lo : required iff strategy != COLLAGE_BF16, else must
+ *   be NULL.   v_lo : required iff strategy == COLLAGE_PLUS, else must be NULL.
+ * Errors: ERR_NULL, ERR_ARG (step 0, bad strategy, hyper range), ERR_ALIAS (overlapping
+ * tensors), ERR_WORKSPACE (edq_out set, workspace too small), ERR_ARCH, ERR_CUDA. */
+collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi, void* v_lo,
+                                    const void* grad, uint64_t n, const collage_hyper_t* hyper,
+                                    uint64_t step, collage_strategy_t strategy, void* stream);
+
+/* Multi-tensor step: all tensors of a plan in ONE launch over a chunk table.
+ * collage_plan_create copies the HOST array `tensors[num]` and builds the device table
+ * (this call allocates and synchronises; do it once, outside the step loop).  chunk_elems is
+ * the work unit handed to a thread block, a multiple of 2048; 0 picks the default.
+ * Tensors with n == 0 are skipped.  The plan records which pointers were NULL; a step whose
+ * strategy needs a missing component fails with ERR_NULL.  EDQ is over all tensors (Eq. 3
+ * with theta the concatenation).
+ * Errors: ERR_NULL, ERR_ARG (num < 0, chunk_elems not a multiple of 2048, more than 2^32-1
+ * chunks), ERR_ALIAS (any two arrays of the plan overlap), ERR_CUDA. */
+collage_status_t collage_plan_create(const collage_tensor_t* tensors, int num, uint32_t chunk_elems,
+                                     collage_plan_t** out_plan);
+collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const collage_hyper_t* hyper,
+                                          uint64_t step, collage_strategy_t strategy, void* stream);
+collage_status_t collage_plan_destroy(collage_plan_t* plan);
+/* Plan facts for callers that report or shard: total elements, number of chunks. */
+uint64_t collage_plan_num_elements(const collage_plan_t* plan);
+uint64_t collage_plan_num_chunks(const collage_plan_t* plan);
+
+/* Batched MCF primitives, elementwise over n bfloat16 values.  Output arrays may be the input
+ * arrays themselves (exact same pointer); partial overlap is ERR_ALIAS.
+ *   fast_two_sum (Theorem 4.1): hi = a (+) b, lo = b (-) (hi (-) a); error-free if |a| >= |b|
+ *   two_sum      (Algorithm TwoSum): same expansion, no ordering needed, 6 operations
+ *   two_prod     (Algorithm TwoProdFMA): hi = a (*) b, lo = fma(a, b, -hi)
+ *   grow         (Algorithm 1): (u, v) = Fast2Sum(x, a); (u, v) = Fast2Sum(u, y (+) v)
+ *   scaling      (Algorithm Scaling): float v times expansion (a1, a2)
+ *   mul          (Algorithm Mul): expansion (a1, a2) times expansion (b1, b2)
+ *   renormalize  (named in the paper's listing keywords, not defined there): Fast2Sum(hi, lo) */
+collage_status_t collage_fast_two_sum(const void* a, const void* b, void* hi, void* lo, uint64_t n, void* stream);
+collage_status_t collage_two_sum(const void* a, const void* b, void* hi, void* lo, uint64_t n, void* stream);
+collage_status_t collage_two_prod(const void* a, const void* b, void* hi, void* lo, uint64_t n, void* stream);
+collage_status_t collage_grow(const void* x, const void* y, const void* a, void* u, void* v, uint64_t n, void* stream);
+collage_status_t collage_scaling(const void* v, const void* a1, const void* a2, void* x, void* e, uint64_t n, void* stream);
+collage_status_t collage_mul(const void* a1, const void* a2, const void* b1, const void* b2, void* x, void* e,
+                             uint64_t n, void* stream);
+collage_status_t collage_renormalize(const void* hi_in, const void* lo_in, void* hi, void* lo, uint64_t n, void* stream);
+
+/* One rounded bfloat16 operation F^BF16(a op b) elementwise (Section 3.1), realised exactly as
+ * inside the step kernel.  op: 0 add, 1 sub, 2 mul, 3 div, 4 sqrt(a), 5 fma(a,b,c).  b is
+ * ignored for sqrt; c only used by fma (pass NULL otherwise). */
+collage_status_t collage_rounded_op(int op, const void* a, const void* b, const void* c, void* out,
+                                    uint64_t n, void* stream);
+
+/* EDQ on stored arrays (Eq. 2-3): old and new parameter expansions and the intended update.
+ * old_lo/new_lo both NULL = plain bfloat16 parameter.  out_dev: DEVICE collage_edq_t*.
+ * Errors: ERR_NULL, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA. */
+collage_status_t collage_edq(const void* old_hi, const void* old_lo, const void* new_hi,
+                             const void* new_lo, const void* delta, uint64_t n, collage_edq_t* out_dev,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COLLAGE_H_ */

@@ -234,7 +234,10 @@ inline void step_one(bf16& th, bf16* dth, bf16& m, bf16& v, bf16* dv, bf16 g,
     const double d = widen(delta);
     acc.dot += d * eff;
     acc.sumsq += d * d;
-    if (d != 0.0 && eff == 0.0) acc.lost += 1;   // lost arithmetic (Def. 3.2): intended update, nothing applied
+    // lost arithmetic (Def. 3.2; "not updated", Figure 3 left): an update was intended and the stored
+    // parameter (every component, compared as values) is what it was
+    const bool unchanged = widen(th) == widen(th_old) && (!dth || widen(*dth) == widen(dth_old));
+    if (d != 0.0 && unchanged) acc.lost += 1;
     if (delta_out) *delta_out = delta;
 }
 
@@ -362,7 +365,9 @@ void oracle_edq(const uint16_t* old_hi, const uint16_t* old_lo, const uint16_t* 
         const double d = widen(delta[i]);
         tot.dot += d * eff;
         tot.sumsq += d * d;
-        if (d != 0.0 && eff == 0.0) tot.lost += 1;
+        const bool unchanged = widen(new_hi[i]) == widen(old_hi[i]) &&
+                               (!(old_lo && new_lo) || widen(new_lo[i]) == widen(old_lo[i]));
+        if (d != 0.0 && unchanged) tot.lost += 1;
     }
     sums_out[0] = tot.dot;
     sums_out[1] = tot.sumsq;

@@ -1,0 +1,199 @@
+"""Thin ctypes binding of the CUDA library: same names as ``include/collage.h``, argument marshalling only.
+
+Tensors are ``torch.bfloat16`` CUDA tensors (or anything with ``data_ptr()``); torch supplies
+device memory and streams, every step of the computation runs in the library's kernels.
+There is no fallback: if the shared library has not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+_LIB_PATH = Path(__file__).resolve().parent / "libcollage_b200.so"
+
+OK, ERR_NULL, ERR_ARG, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_WORKSPACE = range(7)
+BF16, LIGHT, PLUS = 0, 1, 2
+FLAG_EPS_INSIDE_SQRT = 1
+OP_ADD, OP_SUB, OP_MUL, OP_DIV, OP_SQRT, OP_FMA = range(6)
+SCALAR_NAMES = ("b1", "c1", "b2", "c2", "b2h", "b2l", "bc1", "bc2", "a", "lam", "eps")
+
+EXPORTS = (
+    "collage_status_string", "collage_derive_scalars", "collage_workspace_bytes", "collage_adamw_step",
+    "collage_plan_create", "collage_adamw_step_multi", "collage_plan_destroy", "collage_plan_num_elements",
+    "collage_plan_num_chunks", "collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_grow",
+    "collage_scaling", "collage_mul", "collage_renormalize", "collage_rounded_op", "collage_edq",
+)
+
+
+class Hyper(ctypes.Structure):
+    """collage_hyper_t"""
+    _fields_ = [("lr", ctypes.c_double), ("beta1", ctypes.c_double), ("beta2", ctypes.c_double),
+                ("eps", ctypes.c_double), ("weight_decay", ctypes.c_double), ("flags", ctypes.c_uint32),
+                ("edq_out", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+
+
+class Edq(ctypes.Structure):
+    """collage_edq_t"""
+    _fields_ = [("dot", ctypes.c_double), ("sumsq", ctypes.c_double), ("edq", ctypes.c_double),
+                ("n", ctypes.c_uint64), ("lost", ctypes.c_uint64)]
+
+
+class Tensor(ctypes.Structure):
+    """collage_tensor_t"""
+    _fields_ = [("x_hi", ctypes.c_void_p), ("x_lo", ctypes.c_void_p), ("m", ctypes.c_void_p),
+                ("v_hi", ctypes.c_void_p), ("v_lo", ctypes.c_void_p), ("grad", ctypes.c_void_p),
+                ("n", ctypes.c_uint64)]
+
+
+class CollageError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: status {status} ({status_string(status)})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded CUDA library; raises if it has not been built (there is no other path)."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2405_03637_b200.build` "
+                               "(this package has no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(str(_LIB_PATH))
+        vp, u64, i32 = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_int
+        L.collage_status_string.restype = ctypes.c_char_p
+        L.collage_status_string.argtypes = [i32]
+        L.collage_derive_scalars.argtypes = [ctypes.POINTER(Hyper), u64, ctypes.POINTER(ctypes.c_uint16)]
+        L.collage_workspace_bytes.restype = ctypes.c_size_t
+        L.collage_workspace_bytes.argtypes = [u64]
+        L.collage_adamw_step.argtypes = [vp, vp, vp, vp, vp, vp, u64, ctypes.POINTER(Hyper), u64, i32, vp]
+        L.collage_plan_create.argtypes = [ctypes.POINTER(Tensor), i32, ctypes.c_uint32, ctypes.POINTER(vp)]
+        L.collage_adamw_step_multi.argtypes = [vp, ctypes.POINTER(Hyper), u64, i32, vp]
+        L.collage_plan_destroy.argtypes = [vp]
+        L.collage_plan_num_elements.restype = u64
+        L.collage_plan_num_elements.argtypes = [vp]
+        L.collage_plan_num_chunks.restype = u64
+        L.collage_plan_num_chunks.argtypes = [vp]
+        for name in ("collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_renormalize"):
+            getattr(L, name).argtypes = [vp, vp, vp, vp, u64, vp]
+        L.collage_grow.argtypes = [vp, vp, vp, vp, vp, u64, vp]
+        L.collage_scaling.argtypes = [vp, vp, vp, vp, vp, u64, vp]
+        L.collage_mul.argtypes = [vp, vp, vp, vp, vp, vp, u64, vp]
+        L.collage_rounded_op.argtypes = [i32, vp, vp, vp, vp, u64, vp]
+        L.collage_edq.argtypes = [vp, vp, vp, vp, vp, u64, vp, vp, ctypes.c_size_t, vp]
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "cuda_stream"):      # torch.cuda.Stream
+        return t.cuda_stream
+    return t.data_ptr()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise CollageError(status, where)
+
+
+def status_string(status: int) -> str:
+    return lib().collage_status_string(int(status)).decode()
+
+
+def make_hyper(lr, beta1, beta2, eps, weight_decay, flags=0, edq_out=None, workspace=None) -> Hyper:
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    return Hyper(lr, beta1, beta2, eps, weight_decay, flags, _ptr(edq_out), _ptr(workspace), ws_bytes)
+
+
+def derive_scalars(hyper: Hyper, step: int) -> dict:
+    out = (ctypes.c_uint16 * 11)()
+    _check(lib().collage_derive_scalars(ctypes.byref(hyper), step, out), "collage_derive_scalars")
+    return dict(zip(SCALAR_NAMES, (int(v) for v in out)))
+
+
+def workspace_bytes(n_total: int = 0) -> int:
+    return int(lib().collage_workspace_bytes(n_total))
+
+
+def adamw_step(x_hi, x_lo, m, v_hi, v_lo, grad, n, hyper: Hyper, step: int, strategy: int, stream=None):
+    _check(lib().collage_adamw_step(_ptr(x_hi), _ptr(x_lo), _ptr(m), _ptr(v_hi), _ptr(v_lo), _ptr(grad), n,
+                                    ctypes.byref(hyper), step, strategy, _ptr(stream)), "collage_adamw_step")
+
+
+def plan_create(tensors, chunk_elems: int = 0) -> int:
+    """tensors: list of (x_hi, x_lo, m, v_hi, v_lo, grad, n); returns the opaque plan handle."""
+    arr = (Tensor * max(len(tensors), 1))()
+    for i, (x_hi, x_lo, m, v_hi, v_lo, grad, n) in enumerate(tensors):
+        arr[i] = Tensor(_ptr(x_hi), _ptr(x_lo), _ptr(m), _ptr(v_hi), _ptr(v_lo), _ptr(grad), n)
+    plan = ctypes.c_void_p()
+    _check(lib().collage_plan_create(arr, len(tensors), chunk_elems, ctypes.byref(plan)), "collage_plan_create")
+    return plan.value
+
+
+def adamw_step_multi(plan: int, hyper: Hyper, step: int, strategy: int, stream=None):
+    _check(lib().collage_adamw_step_multi(plan, ctypes.byref(hyper), step, strategy, _ptr(stream)),
+           "collage_adamw_step_multi")
+
+
+def plan_destroy(plan: int):
+    _check(lib().collage_plan_destroy(plan), "collage_plan_destroy")
+
+
+def plan_num_elements(plan: int) -> int:
+    return int(lib().collage_plan_num_elements(plan))
+
+
+def plan_num_chunks(plan: int) -> int:
+    return int(lib().collage_plan_num_chunks(plan))
+
+
+def fast_two_sum(a, b, hi, lo, n, stream=None):
+    _check(lib().collage_fast_two_sum(_ptr(a), _ptr(b), _ptr(hi), _ptr(lo), n, _ptr(stream)), "collage_fast_two_sum")
+
+
+def two_sum(a, b, hi, lo, n, stream=None):
+    _check(lib().collage_two_sum(_ptr(a), _ptr(b), _ptr(hi), _ptr(lo), n, _ptr(stream)), "collage_two_sum")
+
+
+def two_prod(a, b, hi, lo, n, stream=None):
+    _check(lib().collage_two_prod(_ptr(a), _ptr(b), _ptr(hi), _ptr(lo), n, _ptr(stream)), "collage_two_prod")
+
+
+def renormalize(hi_in, lo_in, hi, lo, n, stream=None):
+    _check(lib().collage_renormalize(_ptr(hi_in), _ptr(lo_in), _ptr(hi), _ptr(lo), n, _ptr(stream)),
+           "collage_renormalize")
+
+
+def grow(x, y, a, u, v, n, stream=None):
+    _check(lib().collage_grow(_ptr(x), _ptr(y), _ptr(a), _ptr(u), _ptr(v), n, _ptr(stream)), "collage_grow")
+
+
+def scaling(v, a1, a2, x, e, n, stream=None):
+    _check(lib().collage_scaling(_ptr(v), _ptr(a1), _ptr(a2), _ptr(x), _ptr(e), n, _ptr(stream)), "collage_scaling")
+
+
+def mul(a1, a2, b1, b2, x, e, n, stream=None):
+    _check(lib().collage_mul(_ptr(a1), _ptr(a2), _ptr(b1), _ptr(b2), _ptr(x), _ptr(e), n, _ptr(stream)), "collage_mul")
+
+
+def rounded_op(op, a, b, c, out, n, stream=None):
+    _check(lib().collage_rounded_op(op, _ptr(a), _ptr(b), _ptr(c), _ptr(out), n, _ptr(stream)), "collage_rounded_op")
+
+
+def edq(old_hi, old_lo, new_hi, new_lo, delta, n, out_dev, workspace, stream=None):
+    ws_bytes = workspace.numel() * workspace.element_size()
+    _check(lib().collage_edq(_ptr(old_hi), _ptr(old_lo), _ptr(new_hi), _ptr(new_lo), _ptr(delta), n, _ptr(out_dev),
+                             _ptr(workspace), ws_bytes, _ptr(stream)), "collage_edq")
+
+
+def read_edq(edq_dev) -> dict:
+    """Copy a device collage_edq_t (a >= 40-byte torch.uint8 CUDA tensor) to the host and decode it."""
+    raw = edq_dev.detach().cpu().numpy().tobytes()
+    rec = Edq.from_buffer_copy(raw[:ctypes.sizeof(Edq)])
+    return dict(dot=rec.dot, sumsq=rec.sumsq, edq=rec.edq, n=int(rec.n), lost=int(rec.lost))

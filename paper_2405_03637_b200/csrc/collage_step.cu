@@ -1,0 +1,548 @@
+// Fused Collage AdamW step (Algorithm 2 lines 8-13 + EDQ, Eq. 2-3): one persistent kernel that
+// streams every state array exactly once, plus the entry points that launch it.
+//
+// Work is cut into chunks of `chunk_elems` consecutive elements of one tensor.  Thread block b
+// takes chunks b, b + grid, b + 2*grid, ...  Inside a chunk each thread owns 8 consecutive
+// elements (one 16-byte vector per state array) at a time.  Tensors whose pointers are not all
+// 16-byte aligned, and the last (<8) elements of a tensor, go through an element-wise path that
+// feeds the same arithmetic.  EDQ sums: float within a vector, double per thread, fixed-order
+// tree per block, one partial per block, summed by a one-block finalize kernel.
+#include "host_common.cuh"
+#include "mcf_device.cuh"
+
+namespace collage {
+
+constexpr int kThreads = 256;
+constexpr uint32_t kDefaultChunk = 16384;
+
+struct TensorRec {
+    uint16_t* x_hi;
+    uint16_t* x_lo;
+    uint16_t* m;
+    uint16_t* v_hi;
+    uint16_t* v_lo;
+    const uint16_t* grad;
+    uint64_t n;
+    uint32_t aligned;   // all present pointers are 16-byte aligned
+    uint32_t pad;
+};
+
+struct ChunkRec {
+    uint32_t tensor;
+    uint32_t index;     // chunk number inside the tensor: elements [index*chunk_elems, ...)
+};
+
+struct StepParams {
+    TensorRec flat;             // used when the kernel is instantiated FLAT
+    const TensorRec* tensors;   // multi-tensor table (device)
+    const ChunkRec* chunks;     // chunk table (device)
+    uint64_t num_chunks;
+    uint32_t chunk_elems;
+    StepScalars k;
+    EdqPartial* partials;       // one per block, or nullptr
+};
+
+// ---- 16-byte streaming accesses (each byte is touched once: do not keep it in L1) ----------
+__device__ __forceinline__ uint4 ld_stream(const uint16_t* p) {
+    return __ldcs(reinterpret_cast<const uint4*>(p));
+}
+__device__ __forceinline__ void st_stream(uint16_t* p, const uint4& v) {
+    __stcs(reinterpret_cast<uint4*>(p), v);
+}
+
+// element-wise gather/scatter of up to 8 bfloat16 values into / out of four packed registers
+__device__ __forceinline__ uint4 ld_elems(const uint16_t* p, int count) {
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+        if (e < count) w[e >> 1] |= static_cast<uint32_t>(p[e]) << (16 * (e & 1));
+    return make_uint4(w[0], w[1], w[2], w[3]);
+}
+__device__ __forceinline__ void st_elems(uint16_t* p, const uint4& v, int count) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int e = 0; e < 8; ++e)
+        if (e < count) p[e] = static_cast<uint16_t>(w[e >> 1] >> (16 * (e & 1)));
+}
+
+struct Vec {
+    uint4 th, dth, m, v, dv, g;
+};
+
+// The arithmetic of 8 parameters held in registers.  `valid` < 8 masks padded lanes out of EDQ.
+template <int STRATEGY, bool EDQ>
+__device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int valid, double& dot, double& sq,
+                                            uint32_t& lost) {
+    uint32_t* th = reinterpret_cast<uint32_t*>(&s.th);
+    uint32_t* dth = reinterpret_cast<uint32_t*>(&s.dth);
+    uint32_t* m = reinterpret_cast<uint32_t*>(&s.m);
+    uint32_t* v = reinterpret_cast<uint32_t*>(&s.v);
+    uint32_t* dv = reinterpret_cast<uint32_t*>(&s.dv);
+    const uint32_t* g = reinterpret_cast<const uint32_t*>(&s.g);
+    EdqAcc acc = {0.0f, 0.0f, 0u};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        ElemState e;
+        e.th = th[j];
+        e.dth = STRATEGY >= 1 ? dth[j] : 0u;
+        e.m = m[j];
+        e.v = v[j];
+        e.dv = STRATEGY == 2 ? dv[j] : 0u;
+        const bf2 th_old = e.th, dth_old = e.dth;
+        bf2 delta = adamw_pair<STRATEGY>(e, g[j], k);
+        th[j] = e.th;
+        m[j] = e.m;
+        v[j] = e.v;
+        if (STRATEGY >= 1) dth[j] = e.dth;
+        if (STRATEGY == 2) dv[j] = e.dv;
+        if (EDQ) {
+            bf2 th_new = e.th, dth_new = e.dth;
+            if (valid < 8) {            // padded lanes hold zeros on input; keep them out of the sums
+                const int lanes = valid - 2 * j;
+                const uint32_t mask = lanes >= 2 ? 0xFFFFFFFFu : (lanes == 1 ? 0x0000FFFFu : 0u);
+                delta &= mask;
+                th_new &= mask;
+                dth_new &= mask;
+            }
+            edq_pair<(STRATEGY >= 1)>(acc, th_old, dth_old, th_new, dth_new, delta);
+        }
+    }
+    if (EDQ) {
+        dot += static_cast<double>(acc.dot);
+        sq += static_cast<double>(acc.sq);
+        lost += acc.lost;
+    }
+}
+
+template <int STRATEGY>
+__device__ __forceinline__ void load_vec(Vec& s, const TensorRec& t, uint64_t off) {
+    s.th = ld_stream(t.x_hi + off);
+    s.m = ld_stream(t.m + off);
+    s.v = ld_stream(t.v_hi + off);
+    s.g = ld_stream(t.grad + off);
+    if (STRATEGY >= 1) s.dth = ld_stream(t.x_lo + off);
+    if (STRATEGY == 2) s.dv = ld_stream(t.v_lo + off);
+}
+template <int STRATEGY>
+__device__ __forceinline__ void store_vec(const Vec& s, const TensorRec& t, uint64_t off) {
+    st_stream(t.x_hi + off, s.th);
+    st_stream(t.m + off, s.m);
+    st_stream(t.v_hi + off, s.v);
+    if (STRATEGY >= 1) st_stream(t.x_lo + off, s.dth);
+    if (STRATEGY == 2) st_stream(t.v_lo + off, s.dv);
+}
+template <int STRATEGY>
+__device__ __forceinline__ void load_elems(Vec& s, const TensorRec& t, uint64_t off, int count) {
+    s.th = ld_elems(t.x_hi + off, count);
+    s.m = ld_elems(t.m + off, count);
+    s.v = ld_elems(t.v_hi + off, count);
+    s.g = ld_elems(t.grad + off, count);
+    if (STRATEGY >= 1) s.dth = ld_elems(t.x_lo + off, count);
+    if (STRATEGY == 2) s.dv = ld_elems(t.v_lo + off, count);
+}
+template <int STRATEGY>
+__device__ __forceinline__ void store_elems(const Vec& s, const TensorRec& t, uint64_t off, int count) {
+    st_elems(t.x_hi + off, s.th, count);
+    st_elems(t.m + off, s.m, count);
+    st_elems(t.v_hi + off, s.v, count);
+    if (STRATEGY >= 1) st_elems(t.x_lo + off, s.dth, count);
+    if (STRATEGY == 2) st_elems(t.v_lo + off, s.dv, count);
+}
+
+template <int STRATEGY, bool EDQ, bool FLAT, int UNROLL>
+__global__ void __launch_bounds__(kThreads) adamw_step_kernel(const __grid_constant__ StepParams p) {
+    double dot = 0.0, sq = 0.0;
+    uint32_t lost = 0;
+    const StepScalars& k = p.k;
+
+    for (uint64_t c = blockIdx.x; c < p.num_chunks; c += gridDim.x) {
+        TensorRec t;
+        uint64_t start;
+        if (FLAT) {
+            t = p.flat;
+            start = c * p.chunk_elems;
+        } else {
+            const ChunkRec cr = p.chunks[c];
+            t = p.tensors[cr.tensor];
+            start = static_cast<uint64_t>(cr.index) * p.chunk_elems;
+        }
+        const uint64_t left = t.n - start;
+        const uint32_t len = left < p.chunk_elems ? static_cast<uint32_t>(left) : p.chunk_elems;
+        const uint32_t nvec = len >> 3;
+        const int rem = static_cast<int>(len & 7u);
+
+        if (t.aligned) {
+            for (uint32_t i = threadIdx.x; i < nvec; i += kThreads * UNROLL) {
+                Vec s[UNROLL];
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u)
+                    if (i + u * kThreads < nvec) load_vec<STRATEGY>(s[u], t, start + 8ull * (i + u * kThreads));
+#pragma unroll
+                for (int u = 0; u < UNROLL; ++u)
+                    if (i + u * kThreads < nvec) {
+                        compute_vec<STRATEGY, EDQ>(s[u], k, 8, dot, sq, lost);
+                        store_vec<STRATEGY>(s[u], t, start + 8ull * (i + u * kThreads));
+                    }
+            }
+        } else {
+            for (uint32_t i = threadIdx.x; i < nvec; i += kThreads) {
+                Vec s;
+                load_elems<STRATEGY>(s, t, start + 8ull * i, 8);
+                compute_vec<STRATEGY, EDQ>(s, k, 8, dot, sq, lost);
+                store_elems<STRATEGY>(s, t, start + 8ull * i, 8);
+            }
+        }
+        if (rem && threadIdx.x == (nvec % kThreads)) {
+            Vec s;
+            load_elems<STRATEGY>(s, t, start + 8ull * nvec, rem);
+            compute_vec<STRATEGY, EDQ>(s, k, rem, dot, sq, lost);
+            store_elems<STRATEGY>(s, t, start + 8ull * nvec, rem);
+        }
+    }
+
+    if (EDQ) {
+        unsigned long long lost64 = lost;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            dot += __shfl_down_sync(0xFFFFFFFFu, dot, o);
+            sq += __shfl_down_sync(0xFFFFFFFFu, sq, o);
+            lost64 += __shfl_down_sync(0xFFFFFFFFu, lost64, o);
+        }
+        __shared__ double s_dot[kThreads / 32], s_sq[kThreads / 32];
+        __shared__ unsigned long long s_lost[kThreads / 32];
+        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+        if (lane == 0) {
+            s_dot[warp] = dot;
+            s_sq[warp] = sq;
+            s_lost[warp] = lost64;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double d = 0.0, q = 0.0;
+            unsigned long long l = 0;
+#pragma unroll
+            for (int w = 0; w < kThreads / 32; ++w) {
+                d += s_dot[w];
+                q += s_sq[w];
+                l += s_lost[w];
+            }
+            p.partials[blockIdx.x] = EdqPartial{d, q, l, 0ull};
+        }
+    }
+}
+
+// Sums the per-block partials in a fixed order and writes the EDQ record (Eq. 3).
+__global__ void __launch_bounds__(256) edq_finalize_kernel(const EdqPartial* partials, int count, uint64_t n,
+                                                           collage_edq_t* out) {
+    __shared__ double s_dot[256], s_sq[256];
+    __shared__ unsigned long long s_lost[256];
+    double d = 0.0, q = 0.0;
+    unsigned long long l = 0;
+    for (int i = threadIdx.x; i < count; i += 256) {
+        d += partials[i].dot;
+        q += partials[i].sq;
+        l += partials[i].lost;
+    }
+    s_dot[threadIdx.x] = d;
+    s_sq[threadIdx.x] = q;
+    s_lost[threadIdx.x] = l;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) {
+            s_dot[threadIdx.x] += s_dot[threadIdx.x + o];
+            s_sq[threadIdx.x] += s_sq[threadIdx.x + o];
+            s_lost[threadIdx.x] += s_lost[threadIdx.x + o];
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        out->dot = s_dot[0];
+        out->sumsq = s_sq[0];
+        out->edq = s_sq[0] > 0.0 ? s_dot[0] / sqrt(s_sq[0]) : 0.0;
+        out->n = n;
+        out->lost = s_lost[0];
+    }
+}
+
+void launch_edq_finalize(const EdqPartial* partials, int count, uint64_t n, collage_edq_t* out, cudaStream_t stream) {
+    edq_finalize_kernel<<<1, 256, 0, stream>>>(partials, count, n, out);
+}
+
+// ---------------------------------------------------------------- host side ---
+
+static bf2 dup(uint16_t h) { return static_cast<uint32_t>(h) | (static_cast<uint32_t>(h) << 16); }
+
+static collage_status_t make_scalars(const collage_hyper_t* hyper, uint64_t step, StepScalars* k) {
+    uint16_t s[11];
+    const collage_status_t st = collage_derive_scalars(hyper, step, s);
+    if (st != COLLAGE_OK) return st;
+    k->b1 = dup(s[0]);
+    k->c1 = dup(s[1]);
+    k->b2 = dup(s[2]);
+    k->c2 = dup(s[3]);
+    k->b2h = dup(s[4]);
+    k->b2l = dup(s[5]);
+    k->bc1 = dup(s[6]);
+    k->bc2 = dup(s[7]);
+    k->neg_a = dup(s[8] ^ 0x8000u);
+    k->lam = dup(s[9]);
+    k->eps = dup(s[10]);
+    k->flags = hyper->flags;
+    return COLLAGE_OK;
+}
+
+template <int STRATEGY, bool EDQ, bool FLAT>
+static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t stream, int* grid_out) {
+    constexpr int UNROLL = 2;
+    auto kernel = adamw_step_kernel<STRATEGY, EDQ, FLAT, UNROLL>;
+    static int blocks_per_sm = 0;   // per instantiation
+    if (blocks_per_sm == 0) {
+        int b = 0;
+        const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, kThreads, 0);
+        if (e != cudaSuccess) return e;
+        blocks_per_sm = b > 0 ? b : 1;
+    }
+    uint64_t grid = static_cast<uint64_t>(sm_count) * blocks_per_sm;
+    if (grid > p.num_chunks) grid = p.num_chunks;
+    if (grid > static_cast<uint64_t>(kMaxGrid)) grid = kMaxGrid;
+    *grid_out = static_cast<int>(grid);
+    kernel<<<static_cast<unsigned>(grid), kThreads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+template <bool FLAT>
+static cudaError_t dispatch_step(const StepParams& p, int strategy, bool edq, int sm_count, cudaStream_t stream,
+                                 int* grid_out) {
+    switch (strategy * 2 + (edq ? 1 : 0)) {
+        case 0: return launch_step<0, false, FLAT>(p, sm_count, stream, grid_out);
+        case 1: return launch_step<0, true, FLAT>(p, sm_count, stream, grid_out);
+        case 2: return launch_step<1, false, FLAT>(p, sm_count, stream, grid_out);
+        case 3: return launch_step<1, true, FLAT>(p, sm_count, stream, grid_out);
+        case 4: return launch_step<2, false, FLAT>(p, sm_count, stream, grid_out);
+        default: return launch_step<2, true, FLAT>(p, sm_count, stream, grid_out);
+    }
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static collage_status_t check_common(const collage_hyper_t* hyper, uint64_t step, int strategy) {
+    if (!hyper) return COLLAGE_ERR_NULL;
+    if (step == 0) return COLLAGE_ERR_ARG;
+    if (strategy < COLLAGE_BF16 || strategy > COLLAGE_PLUS) return COLLAGE_ERR_ARG;
+    if (!hyper_in_range(hyper)) return COLLAGE_ERR_ARG;
+    if (hyper->flags & ~COLLAGE_FLAG_EPS_INSIDE_SQRT) return COLLAGE_ERR_ARG;
+    if (hyper->edq_out) {
+        if (!hyper->workspace || hyper->workspace_bytes < kWorkspaceBytes) return COLLAGE_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(hyper->workspace) & 15u) return COLLAGE_ERR_WORKSPACE;
+    }
+    return COLLAGE_OK;
+}
+
+}  // namespace collage
+
+using namespace collage;
+
+struct collage_plan {
+    TensorRec* d_tensors = nullptr;
+    ChunkRec* d_chunks = nullptr;
+    uint64_t num_chunks = 0;
+    uint64_t num_elements = 0;
+    uint32_t chunk_elems = 0;
+    int num_tensors = 0;
+    bool has_x_lo = true, has_v_lo = true;
+    int device = 0;
+};
+
+extern "C" {
+
+const char* collage_status_string(collage_status_t status) {
+    switch (status) {
+        case COLLAGE_OK: return "ok";
+        case COLLAGE_ERR_NULL: return "a required pointer is NULL (or a component the strategy needs is missing)";
+        case COLLAGE_ERR_ARG: return "invalid argument (step 0, unknown strategy or op, hyper-parameter out of range)";
+        case COLLAGE_ERR_ALIAS: return "tensors overlap";
+        case COLLAGE_ERR_ARCH: return "current device is not compute capability 10.x (sm_100a only, no fallback)";
+        case COLLAGE_ERR_CUDA: return "CUDA runtime error";
+        case COLLAGE_ERR_WORKSPACE: return "EDQ workspace missing, misaligned or too small";
+    }
+    return "unknown status";
+}
+
+collage_status_t collage_derive_scalars(const collage_hyper_t* hyper, uint64_t step, uint16_t out[11]) {
+    if (!hyper || !out) return COLLAGE_ERR_NULL;
+    if (step == 0 || !hyper_in_range(hyper)) return COLLAGE_ERR_ARG;
+    const double t = static_cast<double>(step);
+    out[0] = double_to_bf16_rn(hyper->beta1);
+    out[1] = double_to_bf16_rn(1.0 - hyper->beta1);
+    out[2] = double_to_bf16_rn(hyper->beta2);
+    out[3] = double_to_bf16_rn(1.0 - hyper->beta2);
+    out[4] = out[2];
+    out[5] = double_to_bf16_rn(hyper->beta2 - bf16_to_double(out[4]));
+    out[6] = double_to_bf16_rn(1.0 - std::pow(hyper->beta1, t));
+    out[7] = double_to_bf16_rn(1.0 - std::pow(hyper->beta2, t));
+    out[8] = double_to_bf16_rn(hyper->lr);
+    out[9] = double_to_bf16_rn(hyper->weight_decay);
+    out[10] = double_to_bf16_rn(hyper->eps);
+    return COLLAGE_OK;
+}
+
+size_t collage_workspace_bytes(uint64_t) { return kWorkspaceBytes; }
+
+collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi, void* v_lo, const void* grad,
+                                    uint64_t n, const collage_hyper_t* hyper, uint64_t step,
+                                    collage_strategy_t strategy, void* stream) {
+    collage_status_t st = check_common(hyper, step, strategy);
+    if (st != COLLAGE_OK) return st;
+    if (!x_hi || !m || !v_hi || !grad) return COLLAGE_ERR_NULL;
+    if ((strategy >= COLLAGE_LIGHT) != (x_lo != nullptr)) return x_lo ? COLLAGE_ERR_ARG : COLLAGE_ERR_NULL;
+    if ((strategy == COLLAGE_PLUS) != (v_lo != nullptr)) return v_lo ? COLLAGE_ERR_ARG : COLLAGE_ERR_NULL;
+    if (n > (1ull << 62)) return COLLAGE_ERR_ARG;
+    std::vector<ByteRange> ranges;
+    for (const void* q : {static_cast<const void*>(x_hi), static_cast<const void*>(x_lo), static_cast<const void*>(m),
+                          static_cast<const void*>(v_hi), static_cast<const void*>(v_lo), grad})
+        push_range(ranges, q, n);
+    if (any_overlap(ranges)) return COLLAGE_ERR_ALIAS;
+    DeviceInfo dev;
+    st = current_device(&dev);
+    if (st != COLLAGE_OK) return st;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+
+    StepParams p{};
+    st = make_scalars(hyper, step, &p.k);
+    if (st != COLLAGE_OK) return st;
+    p.flat.x_hi = static_cast<uint16_t*>(x_hi);
+    p.flat.x_lo = static_cast<uint16_t*>(x_lo);
+    p.flat.m = static_cast<uint16_t*>(m);
+    p.flat.v_hi = static_cast<uint16_t*>(v_hi);
+    p.flat.v_lo = static_cast<uint16_t*>(v_lo);
+    p.flat.grad = static_cast<const uint16_t*>(grad);
+    p.flat.n = n;
+    p.flat.aligned = aligned16(x_hi) && aligned16(x_lo) && aligned16(m) && aligned16(v_hi) && aligned16(v_lo) &&
+                     aligned16(grad);
+    p.chunk_elems = kDefaultChunk;
+    p.num_chunks = (n + kDefaultChunk - 1) / kDefaultChunk;
+    p.partials = static_cast<EdqPartial*>(hyper->workspace);
+    const bool edq = hyper->edq_out != nullptr;
+    int grid = 0;
+    if (n > 0) {
+        if (dispatch_step<true>(p, strategy, edq, dev.sm_count, cs, &grid) != cudaSuccess) return COLLAGE_ERR_CUDA;
+    }
+    if (edq) {
+        launch_edq_finalize(p.partials, grid, n, static_cast<collage_edq_t*>(hyper->edq_out), cs);
+        if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
+    }
+    return COLLAGE_OK;
+}
+
+collage_status_t collage_plan_create(const collage_tensor_t* tensors, int num, uint32_t chunk_elems,
+                                     collage_plan_t** out_plan) {
+    if (!out_plan) return COLLAGE_ERR_NULL;
+    *out_plan = nullptr;
+    if (num < 0) return COLLAGE_ERR_ARG;
+    if (num > 0 && !tensors) return COLLAGE_ERR_NULL;
+    if (chunk_elems == 0) chunk_elems = kDefaultChunk;
+    if (chunk_elems % 2048u) return COLLAGE_ERR_ARG;
+
+    std::vector<TensorRec> recs;
+    std::vector<ChunkRec> chunks;
+    std::vector<ByteRange> ranges;
+    bool has_x_lo = true, has_v_lo = true;
+    uint64_t total = 0;
+    for (int i = 0; i < num; ++i) {
+        const collage_tensor_t& t = tensors[i];
+        if (t.n == 0) continue;
+        if (!t.x_hi || !t.m || !t.v_hi || !t.grad) return COLLAGE_ERR_NULL;
+        if (t.n > (1ull << 62)) return COLLAGE_ERR_ARG;
+        has_x_lo = has_x_lo && t.x_lo;
+        has_v_lo = has_v_lo && t.v_lo;
+        TensorRec r{};
+        r.x_hi = static_cast<uint16_t*>(t.x_hi);
+        r.x_lo = static_cast<uint16_t*>(t.x_lo);
+        r.m = static_cast<uint16_t*>(t.m);
+        r.v_hi = static_cast<uint16_t*>(t.v_hi);
+        r.v_lo = static_cast<uint16_t*>(t.v_lo);
+        r.grad = static_cast<const uint16_t*>(t.grad);
+        r.n = t.n;
+        r.aligned = aligned16(t.x_hi) && aligned16(t.x_lo) && aligned16(t.m) && aligned16(t.v_hi) &&
+                    aligned16(t.v_lo) && aligned16(t.grad);
+        for (const void* q : {static_cast<const void*>(t.x_hi), static_cast<const void*>(t.x_lo),
+                              static_cast<const void*>(t.m), static_cast<const void*>(t.v_hi),
+                              static_cast<const void*>(t.v_lo), t.grad})
+            push_range(ranges, q, t.n);
+        const uint64_t nchunks = (t.n + chunk_elems - 1) / chunk_elems;
+        if (nchunks > 0xFFFFFFFFull || chunks.size() + nchunks > 0xFFFFFFFFull) return COLLAGE_ERR_ARG;
+        const uint32_t id = static_cast<uint32_t>(recs.size());
+        for (uint64_t c = 0; c < nchunks; ++c) chunks.push_back({id, static_cast<uint32_t>(c)});
+        recs.push_back(r);
+        total += t.n;
+    }
+    if (any_overlap(ranges)) return COLLAGE_ERR_ALIAS;
+
+    collage_plan* plan = new collage_plan;
+    plan->num_chunks = chunks.size();
+    plan->num_elements = total;
+    plan->chunk_elems = chunk_elems;
+    plan->num_tensors = static_cast<int>(recs.size());
+    plan->has_x_lo = has_x_lo;
+    plan->has_v_lo = has_v_lo;
+    if (!recs.empty()) {
+        if (cudaGetDevice(&plan->device) != cudaSuccess ||
+            cudaMalloc(&plan->d_tensors, recs.size() * sizeof(TensorRec)) != cudaSuccess ||
+            cudaMalloc(&plan->d_chunks, chunks.size() * sizeof(ChunkRec)) != cudaSuccess ||
+            cudaMemcpy(plan->d_tensors, recs.data(), recs.size() * sizeof(TensorRec), cudaMemcpyHostToDevice) !=
+                cudaSuccess ||
+            cudaMemcpy(plan->d_chunks, chunks.data(), chunks.size() * sizeof(ChunkRec), cudaMemcpyHostToDevice) !=
+                cudaSuccess) {
+            cudaFree(plan->d_tensors);
+            cudaFree(plan->d_chunks);
+            delete plan;
+            return COLLAGE_ERR_CUDA;
+        }
+    }
+    *out_plan = plan;
+    return COLLAGE_OK;
+}
+
+collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const collage_hyper_t* hyper, uint64_t step,
+                                          collage_strategy_t strategy, void* stream) {
+    if (!plan) return COLLAGE_ERR_NULL;
+    collage_status_t st = check_common(hyper, step, strategy);
+    if (st != COLLAGE_OK) return st;
+    if (strategy >= COLLAGE_LIGHT && !plan->has_x_lo) return COLLAGE_ERR_NULL;
+    if (strategy == COLLAGE_PLUS && !plan->has_v_lo) return COLLAGE_ERR_NULL;
+    DeviceInfo dev;
+    st = current_device(&dev);
+    if (st != COLLAGE_OK) return st;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+
+    StepParams p{};
+    st = make_scalars(hyper, step, &p.k);
+    if (st != COLLAGE_OK) return st;
+    p.tensors = plan->d_tensors;
+    p.chunks = plan->d_chunks;
+    p.num_chunks = plan->num_chunks;
+    p.chunk_elems = plan->chunk_elems;
+    p.partials = static_cast<EdqPartial*>(hyper->workspace);
+    const bool edq = hyper->edq_out != nullptr;
+    int grid = 0;
+    if (plan->num_chunks > 0) {
+        if (dispatch_step<false>(p, strategy, edq, dev.sm_count, cs, &grid) != cudaSuccess) return COLLAGE_ERR_CUDA;
+    }
+    if (edq) {
+        launch_edq_finalize(p.partials, grid, plan->num_elements, static_cast<collage_edq_t*>(hyper->edq_out), cs);
+        if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
+    }
+    return COLLAGE_OK;
+}
+
+collage_status_t collage_plan_destroy(collage_plan_t* plan) {
+    if (!plan) return COLLAGE_OK;
+    cudaError_t a = cudaFree(plan->d_tensors), b = cudaFree(plan->d_chunks);
+    delete plan;
+    return (a == cudaSuccess && b == cudaSuccess) ? COLLAGE_OK : COLLAGE_ERR_CUDA;
+}
+
+uint64_t collage_plan_num_elements(const collage_plan_t* plan) { return plan ? plan->num_elements : 0; }
+uint64_t collage_plan_num_chunks(const collage_plan_t* plan) { return plan ? plan->num_chunks : 0; }
+
+}  // extern "C"

@@ -1,0 +1,128 @@
+"""CPU checks of the C-ABI boundary: the library loads, exports what the header declares, derives the
+step's scalars exactly as the oracle does, and rejects bad arguments before touching CUDA."""
+import ctypes
+import re
+from pathlib import Path
+
+import pytest
+
+import oracle
+from paper_2405_03637_b200 import binding as B
+from paper_2405_03637_b200 import build as builder
+
+ROOT = Path(__file__).resolve().parent.parent
+
+
+@pytest.fixture(scope="module")
+def L():
+    builder.build()
+    return B.lib()
+
+
+def test_library_exports_every_declared_symbol(L):
+    header = (ROOT / "include" / "collage.h").read_text()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(collage_[a-z0-9_]+)\s*\(", header))
+    assert declared, "no declarations parsed"
+    assert declared == set(B.EXPORTS)
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_struct_layouts_match_the_header():
+    assert ctypes.sizeof(B.Hyper) == 5 * 8 + 8 + 3 * 8        # flags padded to 8
+    assert ctypes.sizeof(B.Edq) == 40
+    assert ctypes.sizeof(B.Tensor) == 56
+    assert B.workspace_bytes(0) == B.workspace_bytes(1 << 40) > 0
+
+
+@pytest.mark.parametrize("hyp", [
+    dict(lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1),
+    dict(lr=1.2e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1),
+    dict(lr=3e-3, beta1=0.8, beta2=0.98, eps=1e-6, weight_decay=0.0),
+    dict(lr=2e-5, beta1=0.0, beta2=0.99, eps=1e-12, weight_decay=1e-2),
+])
+def test_scalars_equal_the_oracles_bit_for_bit(L, hyp):
+    h = B.make_hyper(**hyp)
+    steps = list(range(1, 3000)) + list(range(3000, 100_001, 97)) + [10 ** 6, 10 ** 9]
+    for t in steps:
+        got = B.derive_scalars(h, t)
+        want = oracle.derive_scalars(hyp["lr"], hyp["beta1"], hyp["beta2"], hyp["eps"], hyp["weight_decay"], t)
+        assert got == want, (t, got, want)
+
+
+def test_host_rounder_equals_oracle_on_awkward_doubles(L):
+    # drive the library's double->bfloat16 rounding through the lr slot (any finite value >= 0 is legal)
+    import numpy as np
+    rng = np.random.default_rng(1)
+    vals = np.concatenate([
+        np.ldexp(rng.uniform(1.0, 2.0, 20000), rng.integers(-140, 128, 20000)),
+        np.ldexp(1.0 + (np.arange(0, 512) + 0.5) / 256.0, -3),             # exact midpoints
+        np.ldexp(np.arange(0, 300) / 2.0, -133),                           # subnormal grid and its midpoints
+        [0.0, 2.0 ** -134, 2.0 ** -135, 3.3895313892515355e38, 3.4e38, 1e39],
+    ])
+    for v in vals:
+        h = B.make_hyper(float(v), 0.9, 0.999, 1e-8, 0.1)
+        assert B.derive_scalars(h, 1)["a"] == oracle.round_to_bf16(float(v)), v
+
+
+def test_argument_errors_are_reported_before_any_cuda_call(L):
+    ok = B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1)
+    dummy = 0x10000  # never dereferenced: every call below must fail validation first
+    call = lambda **kw: L.collage_adamw_step(kw.get("x_hi", dummy), kw.get("x_lo", None), kw.get("m", dummy * 2),
+                                             kw.get("v_hi", dummy * 3), kw.get("v_lo", None), kw.get("grad", dummy * 4),
+                                             kw.get("n", 16), ctypes.byref(kw.get("hyper", ok)), kw.get("step", 1),
+                                             kw.get("strategy", B.BF16), None)
+    assert L.collage_adamw_step(dummy, None, dummy, dummy, None, dummy, 16, None, 1, 0, None) == B.ERR_NULL
+    assert call(step=0) == B.ERR_ARG
+    assert call(strategy=3) == B.ERR_ARG
+    assert call(strategy=-1) == B.ERR_ARG
+    for bad in (dict(lr=-1.0), dict(beta1=1.0), dict(beta2=1.5), dict(eps=float("nan")), dict(weight_decay=float("inf"))):
+        kw = dict(lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
+        kw.update(bad)
+        assert call(hyper=B.make_hyper(**kw)) == B.ERR_ARG
+    assert call(hyper=B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1, flags=8)) == B.ERR_ARG
+    assert call(x_hi=None) == B.ERR_NULL
+    assert call(grad=None) == B.ERR_NULL
+    assert call(strategy=B.LIGHT) == B.ERR_NULL                      # x_lo missing
+    assert call(strategy=B.PLUS, x_lo=dummy * 5) == B.ERR_NULL       # v_lo missing
+    assert call(strategy=B.BF16, x_lo=dummy * 5) == B.ERR_ARG        # component the strategy does not use
+    assert call(m=dummy + 8) == B.ERR_ALIAS                          # m overlaps x_hi
+    assert call(grad=dummy * 3 + 30) == B.ERR_ALIAS                  # grad overlaps the tail of v_hi
+    # EDQ requested without workspace
+    h = B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1)
+    h.edq_out = dummy * 7
+    assert call(hyper=h) == B.ERR_WORKSPACE
+    h.workspace, h.workspace_bytes = dummy * 8, 16
+    assert call(hyper=h) == B.ERR_WORKSPACE
+    # derive_scalars
+    out = (ctypes.c_uint16 * 11)()
+    assert L.collage_derive_scalars(None, 1, out) == B.ERR_NULL
+    assert L.collage_derive_scalars(ctypes.byref(ok), 0, out) == B.ERR_ARG
+    # primitives: NULL, unknown op, partial overlap
+    assert L.collage_grow(dummy, dummy * 2, None, dummy * 3, dummy * 4, 8, None) == B.ERR_NULL
+    assert L.collage_rounded_op(9, dummy, dummy * 2, None, dummy * 3, 8, None) == B.ERR_ARG
+    assert L.collage_fast_two_sum(dummy, dummy * 2, dummy + 2, dummy * 3, 8, None) == B.ERR_ALIAS
+    assert L.collage_fast_two_sum(dummy, dummy * 2, dummy * 3, dummy * 3, 8, None) == B.ERR_ALIAS
+    # plan: bad chunk size, NULL member, overlap between two tensors
+    plan = ctypes.c_void_p()
+    t = (B.Tensor * 2)(B.Tensor(dummy, None, dummy * 2, dummy * 3, None, dummy * 4, 64),
+                       B.Tensor(dummy * 5, None, dummy * 6, dummy * 7, None, dummy * 8, 64))
+    assert L.collage_plan_create(t, 2, 1000, ctypes.byref(plan)) == B.ERR_ARG
+    assert L.collage_plan_create(t, -1, 0, ctypes.byref(plan)) == B.ERR_ARG
+    assert L.collage_plan_create(t, 2, 0, None) == B.ERR_NULL
+    t[1].m = None
+    assert L.collage_plan_create(t, 2, 0, ctypes.byref(plan)) == B.ERR_NULL
+    t[1].m = dummy + 64
+    assert L.collage_plan_create(t, 2, 0, ctypes.byref(plan)) == B.ERR_ALIAS
+    assert L.collage_adamw_step_multi(None, ctypes.byref(ok), 1, 0, None) == B.ERR_NULL
+    assert L.collage_plan_destroy(None) == B.OK
+    for s in range(7):
+        assert B.status_string(s)
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "_lib", None)
+    monkeypatch.setattr(B, "_LIB_PATH", tmp_path / "absent.so")
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        B.lib()

@@ -1,0 +1,115 @@
+"""GPU parity of the one-launch multi-tensor step (chunk table) against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import EdqBuffers, Guarded, assert_same_bits, edq_close, oracle_state, oracle_step
+from paper_2405_03637_b200 import binding as B
+from paper_2405_03637_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+KEYS = ("x_hi", "x_lo", "m", "v_hi", "v_lo")
+
+
+def _build(shapes, strategy, seed, misalign_of=lambda i: 0):
+    """Per-tensor oracle state + guarded device copies + plan."""
+    host, dev, grads = [], [], []
+    for i, (_, n) in enumerate(shapes):
+        theta = W.bits(W.flat_weights(n, seed * 1000 + i)) if n else np.zeros(0, np.uint16)
+        st = oracle_state(theta, strategy)
+        host.append(st)
+        dev.append({k: (Guarded(v, misalign_of(i)) if v is not None else None) for k, v in st.items()})
+        grads.append(Guarded(np.zeros(n, np.uint16), misalign_of(i)))
+    rows = [(d["x_hi"].t, d["x_lo"].t if d["x_lo"] else None, d["m"].t, d["v_hi"].t, d["v_lo"].t if d["v_lo"] else None,
+             g.t, s[1]) for d, g, s in zip(dev, grads, shapes)]
+    return host, dev, grads, rows
+
+
+def _set_grads(shapes, grads, seed, t):
+    out = []
+    for i, (_, n) in enumerate(shapes):
+        g = W.bits(W.flat_grads(n, seed * 1000 + i, t)) if n else np.zeros(0, np.uint16)
+        if n:
+            grads[i].t.copy_(W.from_bits(g, "cuda"))
+        out.append(g)
+    return out
+
+
+def _oracle_multi(host, gbits, t, strategy, hyp):
+    tot = dict(dot=0.0, sumsq=0.0, lost=0)
+    for st, g in zip(host, gbits):
+        if g.size == 0:
+            continue
+        s = oracle_step(st, g, t, strategy, hyp)
+        tot["dot"] += s["dot"]; tot["sumsq"] += s["sumsq"]; tot["lost"] += s["lost"]
+    tot["edq"] = tot["dot"] / np.sqrt(tot["sumsq"]) if tot["sumsq"] > 0 else 0.0
+    return tot
+
+
+@pytest.mark.parametrize("strategy", [0, 1, 2])
+@pytest.mark.parametrize("chunk", [0, 2048, 65536])
+def test_ragged_tensor_set(strategy, chunk):
+    shapes = W.ragged_shapes()
+    hyp = W.HYPERS
+    host, dev, grads, rows = _build(shapes, strategy, seed=3, misalign_of=lambda i: (0, 0, 1, 0, 0, 3)[i % 6])
+    plan = B.plan_create(rows, chunk)
+    assert B.plan_num_elements(plan) == sum(n for _, n in shapes)
+    ce = chunk or 16384
+    assert B.plan_num_chunks(plan) == sum(-(-n // ce) for _, n in shapes)
+    e = EdqBuffers()
+    for t in (1, 2, 3):
+        gbits = _set_grads(shapes, grads, 3, t)
+        B.adamw_step_multi(plan, e.hyper(hyp), t, strategy)
+        torch.cuda.synchronize()
+        want = _oracle_multi(host, gbits, t, strategy, hyp)
+        for i, (st, d) in enumerate(zip(host, dev)):
+            for k in KEYS:
+                if st[k] is not None:
+                    assert_same_bits(d[k].bits(), st[k], f"tensor {i} {k} step {t}")
+                    assert d[k].guards_intact()
+        got = e.read()
+        edq_close(got, want)
+        assert got["n"] == sum(n for _, n in shapes)
+    B.plan_destroy(plan)
+
+
+def test_gpt2_small_shaped_set_collage_light():
+    # 148 tensors, 124,439,808 parameters: whole-array parity for the first steps
+    shapes = W.gpt2_small_shapes()
+    strategy, hyp = 1, W.HYPERS
+    host, dev, grads, rows = _build(shapes, strategy, seed=1)
+    plan = B.plan_create(rows)
+    e = EdqBuffers()
+    for t in (1, 2):
+        gbits = _set_grads(shapes, grads, 1, t)
+        B.adamw_step_multi(plan, e.hyper(hyp), t, strategy)
+        torch.cuda.synchronize()
+        want = _oracle_multi(host, gbits, t, strategy, hyp)
+        for i, (st, d) in enumerate(zip(host, dev)):
+            for k in ("x_hi", "x_lo", "m", "v_hi"):
+                assert_same_bits(d[k].bits(), st[k], f"{shapes[i][0]} {k} step {t}")
+        edq_close(e.read(), want)
+    assert all(d[k].guards_intact() for d in dev for k in ("x_hi", "x_lo", "m", "v_hi"))
+    B.plan_destroy(plan)
+
+
+def test_plan_strategy_needs_its_components():
+    n = 4096
+    z = lambda: torch.zeros(n, dtype=torch.bfloat16, device="cuda")
+    keep = [z() for _ in range(4)]
+    plan = B.plan_create([(keep[0], None, keep[1], keep[2], None, keep[3], n)])
+    h = B.make_hyper(**W.HYPERS)
+    B.adamw_step_multi(plan, h, 1, B.BF16)
+    for s in (B.LIGHT, B.PLUS):
+        with pytest.raises(B.CollageError) as err:
+            B.adamw_step_multi(plan, h, 1, s)
+        assert err.value.status == B.ERR_NULL
+    torch.cuda.synchronize()
+    B.plan_destroy(plan)
+    empty = B.plan_create([])
+    e = EdqBuffers()
+    B.adamw_step_multi(empty, e.hyper(W.HYPERS), 1, B.BF16)
+    torch.cuda.synchronize()
+    assert e.read()["edq"] == 0.0 and e.read()["n"] == 0
+    B.plan_destroy(empty)
