@@ -78,8 +78,26 @@ inline bf16 op_sub(bf16 a, bf16 b) { return round_to_bf16(widen(a) - widen(b)); 
 inline bf16 op_mul(bf16 a, bf16 b) { return round_to_bf16(widen(a) * widen(b)); }
 inline bf16 op_div(bf16 a, bf16 b) { return round_to_bf16(widen(a) / widen(b)); }
 inline bf16 op_sqrt(bf16 a)        { return round_to_bf16(std::sqrt(widen(a))); }
-// a*b + c with a single rounding ("in FMA", Algorithm TwoProdFMA).
-inline bf16 op_fma(bf16 a, bf16 b, bf16 c) { return round_to_bf16(std::fma(widen(a), widen(b), widen(c))); }
+// a*b + c with a single rounding ("in FMA", Algorithm TwoProdFMA).  The product is exact in
+// double; the sum p + c may need far more than 53 bits (a huge product and a tiny addend that only
+// breaks a tie), so it is rounded to odd first: the double keeps a sticky last bit, which makes
+// the final rounding to 8 bits the single rounding of the exact value.
+inline bf16 op_fma(bf16 a, bf16 b, bf16 c) {
+    const double p = widen(a) * widen(b);
+    const double q = widen(c);
+    double s = p + q;
+    if (std::isfinite(s) && std::isfinite(p) && std::isfinite(q)) {
+        const double qv = s - p;
+        const double err = (p - (s - qv)) + (q - qv);      // TwoSum: p + q = s + err exactly
+        if (err != 0.0) {
+            uint64_t bits;
+            std::memcpy(&bits, &s, sizeof bits);
+            if ((bits & 1u) == 0)                           // even: step to the odd neighbour on err's side
+                s = std::nextafter(s, err > 0.0 ? INFINITY : -INFINITY);
+        }
+    }
+    return round_to_bf16(s);
+}
 inline bf16 op_neg(bf16 a) { return a ^ 0x8000u; }
 
 struct pair16 { bf16 hi, lo; };

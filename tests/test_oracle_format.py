@@ -204,6 +204,31 @@ def test_fma_single_rounding_window():
     assert int(oracle.binary_op(oracle.OP_ADD, prod, neg)[0]) == 0
 
 
+def test_fma_is_one_rounding_even_when_the_addend_is_far_below_the_product():
+    # a*b lands exactly on a midpoint of two bfloat16 values; an addend 60 binades below decides the direction.
+    # Rounding the sum to double first would lose the addend and fall back to ties-to-even.
+    a = np.array([0x3F81], np.uint16)                      # 1 + 2^-7
+    b = np.array([0x3FC0], np.uint16)                      # 1.5 -> product 1.5 + 1.5*2^-7 = 1.51171875 (midpoint)
+    lo, hi = 0x3FC1, 0x3FC2                                # neighbours 1.5078125 and 1.515625
+    assert bits_to_f64(a)[0] * bits_to_f64(b)[0] == (bits_to_f64(np.array([lo], np.uint16))[0] +
+                                                     bits_to_f64(np.array([hi], np.uint16))[0]) / 2
+    tiny = oracle.round_to_bf16(2.0 ** -70)
+    up = oracle.binary_op(oracle.OP_FMA, a, b, np.array([tiny], np.uint16))
+    down = oracle.binary_op(oracle.OP_FMA, a, b, np.array([tiny | 0x8000], np.uint16))
+    tie = oracle.binary_op(oracle.OP_FMA, a, b, np.array([0], np.uint16))
+    assert (int(up[0]), int(down[0]), int(tie[0])) == (hi, lo, hi)           # tie itself goes to even (0x3FC2)
+    # brute force against exact rationals over wide exponent ranges, subnormals included
+    rnd = random.Random(23)
+    pool = [int(x) for x in np.concatenate([bf16_window(-126, 100), np.arange(1, 128, dtype=np.uint16)])]
+    trip = [(rnd.choice(pool), rnd.choice(pool), rnd.choice(pool)) for _ in range(20000)]
+    trip = [(x, y, z) for x, y, z in trip if abs(R.decode(x) * R.decode(y)) < 2 ** 120]
+    A, B, C = (np.array(t, np.uint16) for t in zip(*trip))
+    got = oracle.binary_op(oracle.OP_FMA, A, B, C)
+    for (x, y, z), g in zip(trip, got):
+        want = R.fma(x, y, z)
+        assert int(g) == want or ((int(g) | want) & 0x7FFF) == 0, (hex(x), hex(y), hex(z), hex(int(g)), hex(want))
+
+
 def test_ulp_helper_matches_definition():
     # Def. 3.1 with the paper's examples: ulp(1) = 2^-7, ulp(200) = 1, subnormals share 2^-133
     assert ulp_f64(np.array([0x3F80], np.uint16))[0] == 2.0 ** -7
