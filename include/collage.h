@@ -116,6 +116,24 @@ collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi,
                                     const void* grad, uint64_t n, const collage_hyper_t* hyper,
                                     uint64_t step, collage_strategy_t strategy, void* stream);
 
+/* The same step for state that lives in HOST memory (optimizer state kept off the device).
+ * All six tensor pointers are HOST pointers (page-locked memory is needed for the copies to
+ * overlap; pageable memory works, serialised by the runtime).  The arrays are streamed through
+ * `staging_dev`, a DEVICE buffer of `staging_bytes` bytes (256-byte aligned, at least
+ * collage_workspace_bytes() + 1 MiB; larger is faster up to a few hundred MiB), in slabs: while
+ * slab i is computed, slab i+1 is copied in and slab i-1 copied out on two internal copy streams
+ * that the library creates per device on the first call.  Work is ordered after earlier work on
+ * `stream`, and `stream` waits for the last copy-out, so synchronising `stream` suffices.
+ * hyper->edq_out, if set, is a HOST collage_edq_t* here (written by a copy enqueued on
+ * `stream`); hyper->workspace is ignored.  Results are bit-identical to collage_adamw_step.
+ * Calls on one device share the copy streams: issue them one at a time per device.
+ * Errors: as collage_adamw_step, with ERR_WORKSPACE for a missing, misaligned or too small
+ * staging buffer. */
+collage_status_t collage_adamw_step_host(void* x_hi, void* x_lo, void* m, void* v_hi, void* v_lo,
+                                         const void* grad, uint64_t n, const collage_hyper_t* hyper,
+                                         uint64_t step, collage_strategy_t strategy, void* staging_dev,
+                                         size_t staging_bytes, void* stream);
+
 /* Multi-tensor step: all tensors of a plan in ONE launch over a chunk table.
  * collage_plan_create copies the HOST array `tensors[num]` and builds the device table
  * (this call allocates and synchronises; do it once, outside the step loop).  chunk_elems is
@@ -164,6 +182,18 @@ collage_status_t collage_rounded_op(int op, const void* a, const void* b, const 
 collage_status_t collage_edq(const void* old_hi, const void* old_lo, const void* new_hi,
                              const void* new_lo, const void* delta, uint64_t n, collage_edq_t* out_dev,
                              void* workspace, size_t workspace_bytes, void* stream);
+
+/* Exhaustive self test of the arithmetic the kernels rely on, on the current device (Section 3.1's
+ * model: one rounding to nearest-even per operation).  Compares, for EVERY pair of bfloat16 bit
+ * patterns (2^32 pairs; 2^16 values for the root), the realisation used in the kernels with a
+ * reference built from IEEE float/double arithmetic and one conversion to bfloat16:
+ *   out_host[0] add  [1] sub  [2] mul            native packed bfloat16 instructions
+ *   out_host[3] div  [4] sqrt                    reciprocal / root approximations vs div.rn, sqrt.rn
+ *   out_host[5] division by a scalar through a host-rounded reciprocal (divisors in (0, 1])
+ * Each entry is the number of results that differ (NaNs compared as a class); all must be 0.
+ * HOST output; allocates a few bytes, synchronises `stream`; takes about a second.
+ * Errors: ERR_NULL, ERR_ARCH, ERR_CUDA. */
+collage_status_t collage_selftest(uint64_t out_host[6], void* stream);
 
 #ifdef __cplusplus
 }

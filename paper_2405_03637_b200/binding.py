@@ -19,9 +19,11 @@ SCALAR_NAMES = ("b1", "c1", "b2", "c2", "b2h", "b2l", "bc1", "bc2", "a", "lam", 
 
 EXPORTS = (
     "collage_status_string", "collage_derive_scalars", "collage_workspace_bytes", "collage_adamw_step",
+    "collage_adamw_step_host",
     "collage_plan_create", "collage_adamw_step_multi", "collage_plan_destroy", "collage_plan_num_elements",
     "collage_plan_num_chunks", "collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_grow",
     "collage_scaling", "collage_mul", "collage_renormalize", "collage_rounded_op", "collage_edq",
+    "collage_selftest",
 )
 
 
@@ -69,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.collage_workspace_bytes.restype = ctypes.c_size_t
         L.collage_workspace_bytes.argtypes = [u64]
         L.collage_adamw_step.argtypes = [vp, vp, vp, vp, vp, vp, u64, ctypes.POINTER(Hyper), u64, i32, vp]
+        L.collage_adamw_step_host.argtypes = [vp, vp, vp, vp, vp, vp, u64, ctypes.POINTER(Hyper), u64, i32, vp,
+                                              ctypes.c_size_t, vp]
         L.collage_plan_create.argtypes = [ctypes.POINTER(Tensor), i32, ctypes.c_uint32, ctypes.POINTER(vp)]
         L.collage_adamw_step_multi.argtypes = [vp, ctypes.POINTER(Hyper), u64, i32, vp]
         L.collage_plan_destroy.argtypes = [vp]
@@ -83,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.collage_mul.argtypes = [vp, vp, vp, vp, vp, vp, u64, vp]
         L.collage_rounded_op.argtypes = [i32, vp, vp, vp, vp, u64, vp]
         L.collage_edq.argtypes = [vp, vp, vp, vp, vp, u64, vp, vp, ctypes.c_size_t, vp]
+        L.collage_selftest.argtypes = [ctypes.POINTER(ctypes.c_uint64), vp]
         _lib = L
     return _lib
 
@@ -124,6 +129,14 @@ def workspace_bytes(n_total: int = 0) -> int:
 def adamw_step(x_hi, x_lo, m, v_hi, v_lo, grad, n, hyper: Hyper, step: int, strategy: int, stream=None):
     _check(lib().collage_adamw_step(_ptr(x_hi), _ptr(x_lo), _ptr(m), _ptr(v_hi), _ptr(v_lo), _ptr(grad), n,
                                     ctypes.byref(hyper), step, strategy, _ptr(stream)), "collage_adamw_step")
+
+
+def adamw_step_host(x_hi, x_lo, m, v_hi, v_lo, grad, n, hyper: Hyper, step: int, strategy: int, staging, stream=None):
+    """Host-resident state (pinned CPU tensors); `staging` is a CUDA uint8 tensor; hyper.edq_out is a host address."""
+    _check(lib().collage_adamw_step_host(_ptr(x_hi), _ptr(x_lo), _ptr(m), _ptr(v_hi), _ptr(v_lo), _ptr(grad), n,
+                                         ctypes.byref(hyper), step, strategy, _ptr(staging),
+                                         staging.numel() * staging.element_size(), _ptr(stream)),
+           "collage_adamw_step_host")
 
 
 def plan_create(tensors, chunk_elems: int = 0) -> int:
@@ -190,6 +203,12 @@ def edq(old_hi, old_lo, new_hi, new_lo, delta, n, out_dev, workspace, stream=Non
     ws_bytes = workspace.numel() * workspace.element_size()
     _check(lib().collage_edq(_ptr(old_hi), _ptr(old_lo), _ptr(new_hi), _ptr(new_lo), _ptr(delta), n, _ptr(out_dev),
                              _ptr(workspace), ws_bytes, _ptr(stream)), "collage_edq")
+
+
+def selftest(stream=None) -> dict:
+    out = (ctypes.c_uint64 * 6)()
+    _check(lib().collage_selftest(out, _ptr(stream)), "collage_selftest")
+    return dict(zip(("add", "sub", "mul", "div", "sqrt", "scalar_div"), (int(v) for v in out)))
 
 
 def read_edq(edq_dev) -> dict:

@@ -6,7 +6,8 @@
 
 namespace collage {
 
-void launch_edq_finalize(const EdqPartial* partials, int count, uint64_t n, collage_edq_t* out, cudaStream_t stream);
+void launch_edq_finalize(const EdqPartial* partials, int count, uint64_t n, collage_edq_t* out, cudaStream_t stream,
+                         bool accumulate);
 
 constexpr int kPrimThreads = 256;
 
@@ -197,11 +198,11 @@ __global__ void __launch_bounds__(kPrimThreads) edq_kernel(const __grid_constant
                     if (e < count) w[a][e >> 1] |= static_cast<uint32_t>(src[a][off + e]) << (16 * (e & 1));
             }
         }
-        EdqAcc acc = {0.0f, 0.0f, 0u};
+        EdqAcc acc = {0ull, 0ull, 0u};
 #pragma unroll
         for (int j = 0; j < 4; ++j) edq_pair<HAS_LO>(acc, w[0][j], w[1][j], w[2][j], w[3][j], w[4][j]);
-        dot += static_cast<double>(acc.dot);
-        sq += static_cast<double>(acc.sq);
+        dot += static_cast<double>(edq_dot(acc));
+        sq += static_cast<double>(edq_sq(acc));
         lost += acc.lost;
     }
 #pragma unroll
@@ -229,6 +230,63 @@ __global__ void __launch_bounds__(kPrimThreads) edq_kernel(const __grid_constant
             l += s_lost[x];
         }
         p.partials[blockIdx.x] = EdqPartial{d, q, l, 0ull};
+    }
+}
+
+// ------------------------------------------------------------- self test ---
+// Exhaustive comparison of the arithmetic realisations used by the kernels with references
+// built from IEEE float/double arithmetic and one cvt.rn to bfloat16.
+
+__device__ __forceinline__ bool same_or_both_nan(uint32_t x, uint32_t y) {
+    const bool xn = (x & 0x7F80u) == 0x7F80u && (x & 0x7Fu), yn = (y & 0x7F80u) == 0x7F80u && (y & 0x7Fu);
+    return x == y || (xn && yn);
+}
+__device__ __forceinline__ uint32_t mismatches(bf2 x, bf2 y) {
+    return (same_or_both_nan(x & 0xFFFFu, y & 0xFFFFu) ? 0u : 1u) + (same_or_both_nan(x >> 16, y >> 16) ? 0u : 1u);
+}
+// exact product of two bfloat16 values rounded once: double product (exact), truncated to float
+// with a sticky last bit (round to odd), then cvt.rn
+__device__ __forceinline__ float product_round_to_odd(float a, float b) {
+    const double p = static_cast<double>(a) * static_cast<double>(b);
+    float f = __double2float_rz(p);
+    if (static_cast<double>(f) != p && isfinite(f)) f = __uint_as_float(__float_as_uint(f) | 1u);
+    return f;
+}
+
+__global__ void __launch_bounds__(256) selftest_kernel(unsigned long long* counts) {
+    unsigned long long c_add = 0, c_sub = 0, c_mul = 0, c_div = 0, c_sdiv = 0;
+    const uint64_t stride = static_cast<uint64_t>(gridDim.x) * blockDim.x;
+    // every (a, b): a in the outer 16 bits, two consecutive b per item
+    for (uint64_t i = blockIdx.x * static_cast<uint64_t>(blockDim.x) + threadIdx.x; i < (1ull << 31); i += stride) {
+        const uint32_t a16 = static_cast<uint32_t>(i >> 15), b16 = static_cast<uint32_t>(i & 0x7FFFu) * 2u;
+        const bf2 a = a16 | (a16 << 16), b = b16 | ((b16 + 1u) << 16);
+        const float a0 = lo_f32(a), a1 = hi_f32(a), b0 = lo_f32(b), b1 = hi_f32(b);
+        c_add += mismatches(add2(a, b), pack_rn(__fadd_rn(a1, b1), __fadd_rn(a0, b0)));
+        c_sub += mismatches(sub2(a, b), pack_rn(__fsub_rn(a1, b1), __fsub_rn(a0, b0)));
+        c_mul += mismatches(mul2(a, b), pack_rn(product_round_to_odd(a1, b1), product_round_to_odd(a0, b0)));
+        c_div += mismatches(div2(a, b), div2_ieee(a, b));
+        // scalar-divisor route: divisors are the positive normal values up to 1 (bias corrections live there)
+        if (b16 >= 0x0080u && b16 + 1u <= 0x3F80u) {
+            const double d0 = static_cast<double>(b0), d1 = static_cast<double>(b1);
+            // the host vouches for divisors in [2^-100, 1]: the reciprocal is then used without any test
+            const float r0 = (d0 >= 0x1p-100) ? static_cast<float>(1.0 / d0) : nanf("");
+            const float r1 = (d1 >= 0x1p-100) ? static_cast<float>(1.0 / d1) : nanf("");
+            const bf2 q0 = div2_scalar(a, b0, r0), q1 = div2_scalar(a, b1, r1);
+            c_sdiv += mismatches((q0 & 0xFFFFu) | (q1 << 16), div2_ieee(a, b));
+        }
+    }
+    unsigned long long c_sqrt = 0;
+    for (uint64_t i = blockIdx.x * static_cast<uint64_t>(blockDim.x) + threadIdx.x; i < (1ull << 15); i += stride) {
+        const uint32_t x = static_cast<uint32_t>(i) * 2u;
+        const bf2 a = x | ((x + 1u) << 16);
+        c_sqrt += mismatches(sqrt2(a), sqrt2_ieee(a));
+    }
+    unsigned long long v[6] = {c_add, c_sub, c_mul, c_div, c_sqrt, c_sdiv};
+#pragma unroll
+    for (int k = 0; k < 6; ++k) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v[k] += __shfl_down_sync(0xFFFFFFFFu, v[k], o);
+        if ((threadIdx.x & 31) == 0 && v[k]) atomicAdd(&counts[k], v[k]);
     }
 }
 
@@ -310,8 +368,27 @@ collage_status_t collage_edq(const void* old_hi, const void* old_lo, const void*
         else edq_kernel<false><<<static_cast<unsigned>(grid), kPrimThreads, 0, cs>>>(p);
         if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
-    launch_edq_finalize(p.partials, static_cast<int>(grid), n, out_dev, cs);
+    launch_edq_finalize(p.partials, static_cast<int>(grid), n, out_dev, cs, false);
     return cudaGetLastError() == cudaSuccess ? COLLAGE_OK : COLLAGE_ERR_CUDA;
+}
+
+collage_status_t collage_selftest(uint64_t out_host[6], void* stream) {
+    if (!out_host) return COLLAGE_ERR_NULL;
+    DeviceInfo dev;
+    const collage_status_t st = current_device(&dev);
+    if (st != COLLAGE_OK) return st;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    unsigned long long* counts = nullptr;
+    if (cudaMalloc(&counts, 6 * sizeof(unsigned long long)) != cudaSuccess) return COLLAGE_ERR_CUDA;
+    cudaError_t e = cudaMemsetAsync(counts, 0, 6 * sizeof(unsigned long long), cs);
+    if (e == cudaSuccess) {
+        selftest_kernel<<<dev.sm_count * 8, 256, 0, cs>>>(counts);
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaMemcpyAsync(out_host, counts, 6 * sizeof(unsigned long long), cudaMemcpyDeviceToHost, cs);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(cs);
+    cudaFree(counts);
+    return e == cudaSuccess ? COLLAGE_OK : COLLAGE_ERR_CUDA;
 }
 
 }  // extern "C"

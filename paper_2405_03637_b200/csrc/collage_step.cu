@@ -12,7 +12,18 @@
 
 namespace collage {
 
-constexpr int kThreads = 256;
+// Launch geometry of the step kernel (measured on B200: 128 threads x 6 resident blocks per SM,
+// one 8-element vector per thread in flight, 80 registers, was the fastest of the shapes tried).
+#ifndef COLLAGE_THREADS
+#define COLLAGE_THREADS 128
+#endif
+#ifndef COLLAGE_UNROLL
+#define COLLAGE_UNROLL 1
+#endif
+#ifndef COLLAGE_MINBLOCKS
+#define COLLAGE_MINBLOCKS 6
+#endif
+constexpr int kThreads = COLLAGE_THREADS;
 constexpr uint32_t kDefaultChunk = 16384;
 
 struct TensorRec {
@@ -70,7 +81,7 @@ struct Vec {
 };
 
 // The arithmetic of 8 parameters held in registers.  `valid` < 8 masks padded lanes out of EDQ.
-template <int STRATEGY, bool EDQ>
+template <int STRATEGY, bool EDQ, bool FAST>
 __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int valid, double& dot, double& sq,
                                             uint32_t& lost) {
     uint32_t* th = reinterpret_cast<uint32_t*>(&s.th);
@@ -79,7 +90,7 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
     uint32_t* v = reinterpret_cast<uint32_t*>(&s.v);
     uint32_t* dv = reinterpret_cast<uint32_t*>(&s.dv);
     const uint32_t* g = reinterpret_cast<const uint32_t*>(&s.g);
-    EdqAcc acc = {0.0f, 0.0f, 0u};
+    EdqAcc acc = {0ull, 0ull, 0u};
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         ElemState e;
@@ -89,7 +100,7 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
         e.v = v[j];
         e.dv = STRATEGY == 2 ? dv[j] : 0u;
         const bf2 th_old = e.th, dth_old = e.dth;
-        bf2 delta = adamw_pair<STRATEGY>(e, g[j], k);
+        bf2 delta = adamw_pair<STRATEGY, FAST>(e, g[j], k);
         th[j] = e.th;
         m[j] = e.m;
         v[j] = e.v;
@@ -108,8 +119,8 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
         }
     }
     if (EDQ) {
-        dot += static_cast<double>(acc.dot);
-        sq += static_cast<double>(acc.sq);
+        dot += static_cast<double>(edq_dot(acc));
+        sq += static_cast<double>(edq_sq(acc));
         lost += acc.lost;
     }
 }
@@ -149,8 +160,8 @@ __device__ __forceinline__ void store_elems(const Vec& s, const TensorRec& t, ui
     if (STRATEGY == 2) st_elems(t.v_lo + off, s.dv, count);
 }
 
-template <int STRATEGY, bool EDQ, bool FLAT, int UNROLL>
-__global__ void __launch_bounds__(kThreads) adamw_step_kernel(const __grid_constant__ StepParams p) {
+template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, int UNROLL>
+__global__ void __launch_bounds__(kThreads, COLLAGE_MINBLOCKS) adamw_step_kernel(const __grid_constant__ StepParams p) {
     double dot = 0.0, sq = 0.0;
     uint32_t lost = 0;
     const StepScalars& k = p.k;
@@ -180,7 +191,7 @@ __global__ void __launch_bounds__(kThreads) adamw_step_kernel(const __grid_const
 #pragma unroll
                 for (int u = 0; u < UNROLL; ++u)
                     if (i + u * kThreads < nvec) {
-                        compute_vec<STRATEGY, EDQ>(s[u], k, 8, dot, sq, lost);
+                        compute_vec<STRATEGY, EDQ, FAST>(s[u], k, 8, dot, sq, lost);
                         store_vec<STRATEGY>(s[u], t, start + 8ull * (i + u * kThreads));
                     }
             }
@@ -188,14 +199,14 @@ __global__ void __launch_bounds__(kThreads) adamw_step_kernel(const __grid_const
             for (uint32_t i = threadIdx.x; i < nvec; i += kThreads) {
                 Vec s;
                 load_elems<STRATEGY>(s, t, start + 8ull * i, 8);
-                compute_vec<STRATEGY, EDQ>(s, k, 8, dot, sq, lost);
+                compute_vec<STRATEGY, EDQ, FAST>(s, k, 8, dot, sq, lost);
                 store_elems<STRATEGY>(s, t, start + 8ull * i, 8);
             }
         }
         if (rem && threadIdx.x == (nvec % kThreads)) {
             Vec s;
             load_elems<STRATEGY>(s, t, start + 8ull * nvec, rem);
-            compute_vec<STRATEGY, EDQ>(s, k, rem, dot, sq, lost);
+            compute_vec<STRATEGY, EDQ, FAST>(s, k, rem, dot, sq, lost);
             store_elems<STRATEGY>(s, t, start + 8ull * nvec, rem);
         }
     }
@@ -232,8 +243,9 @@ __global__ void __launch_bounds__(kThreads) adamw_step_kernel(const __grid_const
 }
 
 // Sums the per-block partials in a fixed order and writes the EDQ record (Eq. 3).
+// With `accumulate` the sums are added to the record's current contents (a step issued in slabs).
 __global__ void __launch_bounds__(256) edq_finalize_kernel(const EdqPartial* partials, int count, uint64_t n,
-                                                           collage_edq_t* out) {
+                                                           collage_edq_t* out, int accumulate) {
     __shared__ double s_dot[256], s_sq[256];
     __shared__ unsigned long long s_lost[256];
     double d = 0.0, q = 0.0;
@@ -256,16 +268,25 @@ __global__ void __launch_bounds__(256) edq_finalize_kernel(const EdqPartial* par
         __syncthreads();
     }
     if (threadIdx.x == 0) {
-        out->dot = s_dot[0];
-        out->sumsq = s_sq[0];
-        out->edq = s_sq[0] > 0.0 ? s_dot[0] / sqrt(s_sq[0]) : 0.0;
+        double dot = s_dot[0], sq = s_sq[0];
+        unsigned long long lost = s_lost[0];
+        if (accumulate) {
+            dot += out->dot;
+            sq += out->sumsq;
+            lost += out->lost;
+            n += out->n;
+        }
+        out->dot = dot;
+        out->sumsq = sq;
+        out->edq = sq > 0.0 ? dot / sqrt(sq) : 0.0;
         out->n = n;
-        out->lost = s_lost[0];
+        out->lost = lost;
     }
 }
 
-void launch_edq_finalize(const EdqPartial* partials, int count, uint64_t n, collage_edq_t* out, cudaStream_t stream) {
-    edq_finalize_kernel<<<1, 256, 0, stream>>>(partials, count, n, out);
+void launch_edq_finalize(const EdqPartial* partials, int count, uint64_t n, collage_edq_t* out, cudaStream_t stream,
+                         bool accumulate) {
+    edq_finalize_kernel<<<1, 256, 0, stream>>>(partials, count, n, out, accumulate ? 1 : 0);
 }
 
 // ---------------------------------------------------------------- host side ---
@@ -282,19 +303,31 @@ static collage_status_t make_scalars(const collage_hyper_t* hyper, uint64_t step
     k->c2 = dup(s[3]);
     k->b2h = dup(s[4]);
     k->b2l = dup(s[5]);
-    k->bc1 = dup(s[6]);
-    k->bc2 = dup(s[7]);
+    // scalar divisors as floats, with a host-rounded reciprocal when it is safely normal
+    auto reciprocal = [](double d) {
+        return (d >= 0x1p-100 && d <= 0x1p100) ? static_cast<float>(1.0 / d) : std::nanf("");
+    };
+    k->bc1 = static_cast<float>(bf16_to_double(s[6]));
+    k->bc2 = static_cast<float>(bf16_to_double(s[7]));
+    k->rbc1 = reciprocal(bf16_to_double(s[6]));
+    k->rbc2 = reciprocal(bf16_to_double(s[7]));
     k->neg_a = dup(s[8] ^ 0x8000u);
     k->lam = dup(s[9]);
     k->eps = dup(s[10]);
     k->flags = hyper->flags;
+    // the lean arithmetic chain of the kernel is valid for these ranges (every practical setting)
+    const double bc1 = bf16_to_double(s[6]), bc2 = bf16_to_double(s[7]), eps = bf16_to_double(s[10]);
+    k->fast = (bc1 >= 0x1p-100 && bc1 <= 1.0 && bc2 >= 0x1p-100 && bc2 <= 1.0 && eps >= 0x1p-54 && eps <= 0x1p60) ? 1u : 0u;
+#ifdef COLLAGE_IEEE_DIV_SQRT
+    k->fast = 0u;
+#endif
     return COLLAGE_OK;
 }
 
-template <int STRATEGY, bool EDQ, bool FLAT>
+template <int STRATEGY, bool EDQ, bool FLAT, bool FAST>
 static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t stream, int* grid_out) {
-    constexpr int UNROLL = 2;
-    auto kernel = adamw_step_kernel<STRATEGY, EDQ, FLAT, UNROLL>;
+    constexpr int UNROLL = COLLAGE_UNROLL;
+    auto kernel = adamw_step_kernel<STRATEGY, EDQ, FLAT, FAST, UNROLL>;
     static int blocks_per_sm = 0;   // per instantiation
     if (blocks_per_sm == 0) {
         int b = 0;
@@ -310,20 +343,49 @@ static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t s
     return cudaGetLastError();
 }
 
+template <bool FLAT, bool FAST>
+static cudaError_t dispatch_step2(const StepParams& p, int strategy, bool edq, int sm_count, cudaStream_t stream,
+                                  int* grid_out) {
+    switch (strategy * 2 + (edq ? 1 : 0)) {
+        case 0: return launch_step<0, false, FLAT, FAST>(p, sm_count, stream, grid_out);
+        case 1: return launch_step<0, true, FLAT, FAST>(p, sm_count, stream, grid_out);
+        case 2: return launch_step<1, false, FLAT, FAST>(p, sm_count, stream, grid_out);
+        case 3: return launch_step<1, true, FLAT, FAST>(p, sm_count, stream, grid_out);
+        case 4: return launch_step<2, false, FLAT, FAST>(p, sm_count, stream, grid_out);
+        default: return launch_step<2, true, FLAT, FAST>(p, sm_count, stream, grid_out);
+    }
+}
 template <bool FLAT>
 static cudaError_t dispatch_step(const StepParams& p, int strategy, bool edq, int sm_count, cudaStream_t stream,
                                  int* grid_out) {
-    switch (strategy * 2 + (edq ? 1 : 0)) {
-        case 0: return launch_step<0, false, FLAT>(p, sm_count, stream, grid_out);
-        case 1: return launch_step<0, true, FLAT>(p, sm_count, stream, grid_out);
-        case 2: return launch_step<1, false, FLAT>(p, sm_count, stream, grid_out);
-        case 3: return launch_step<1, true, FLAT>(p, sm_count, stream, grid_out);
-        case 4: return launch_step<2, false, FLAT>(p, sm_count, stream, grid_out);
-        default: return launch_step<2, true, FLAT>(p, sm_count, stream, grid_out);
-    }
+    return p.k.fast ? dispatch_step2<FLAT, true>(p, strategy, edq, sm_count, stream, grid_out)
+                    : dispatch_step2<FLAT, false>(p, strategy, edq, sm_count, stream, grid_out);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Launches the flat (single tensor) step on device pointers; no-op for n == 0.
+static cudaError_t launch_flat(void* x_hi, void* x_lo, void* m, void* v_hi, void* v_lo, const void* grad, uint64_t n,
+                               const StepScalars& k, int strategy, bool edq, EdqPartial* partials, int sm_count,
+                               cudaStream_t stream, int* grid_out) {
+    *grid_out = 0;
+    if (n == 0) return cudaSuccess;
+    StepParams p{};
+    p.k = k;
+    p.flat.x_hi = static_cast<uint16_t*>(x_hi);
+    p.flat.x_lo = static_cast<uint16_t*>(x_lo);
+    p.flat.m = static_cast<uint16_t*>(m);
+    p.flat.v_hi = static_cast<uint16_t*>(v_hi);
+    p.flat.v_lo = static_cast<uint16_t*>(v_lo);
+    p.flat.grad = static_cast<const uint16_t*>(grad);
+    p.flat.n = n;
+    p.flat.aligned = aligned16(x_hi) && aligned16(x_lo) && aligned16(m) && aligned16(v_hi) && aligned16(v_lo) &&
+                     aligned16(grad);
+    p.chunk_elems = kDefaultChunk;
+    p.num_chunks = (n + kDefaultChunk - 1) / kDefaultChunk;
+    p.partials = partials;
+    return dispatch_step<true>(p, strategy, edq, sm_count, stream, grid_out);
+}
 
 static collage_status_t check_common(const collage_hyper_t* hyper, uint64_t step, int strategy) {
     if (!hyper) return COLLAGE_ERR_NULL;
@@ -407,28 +469,17 @@ collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi,
     if (st != COLLAGE_OK) return st;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
-    StepParams p{};
-    st = make_scalars(hyper, step, &p.k);
+    StepScalars k;
+    st = make_scalars(hyper, step, &k);
     if (st != COLLAGE_OK) return st;
-    p.flat.x_hi = static_cast<uint16_t*>(x_hi);
-    p.flat.x_lo = static_cast<uint16_t*>(x_lo);
-    p.flat.m = static_cast<uint16_t*>(m);
-    p.flat.v_hi = static_cast<uint16_t*>(v_hi);
-    p.flat.v_lo = static_cast<uint16_t*>(v_lo);
-    p.flat.grad = static_cast<const uint16_t*>(grad);
-    p.flat.n = n;
-    p.flat.aligned = aligned16(x_hi) && aligned16(x_lo) && aligned16(m) && aligned16(v_hi) && aligned16(v_lo) &&
-                     aligned16(grad);
-    p.chunk_elems = kDefaultChunk;
-    p.num_chunks = (n + kDefaultChunk - 1) / kDefaultChunk;
-    p.partials = static_cast<EdqPartial*>(hyper->workspace);
     const bool edq = hyper->edq_out != nullptr;
     int grid = 0;
-    if (n > 0) {
-        if (dispatch_step<true>(p, strategy, edq, dev.sm_count, cs, &grid) != cudaSuccess) return COLLAGE_ERR_CUDA;
-    }
+    if (launch_flat(x_hi, x_lo, m, v_hi, v_lo, grad, n, k, strategy, edq, static_cast<EdqPartial*>(hyper->workspace),
+                    dev.sm_count, cs, &grid) != cudaSuccess)
+        return COLLAGE_ERR_CUDA;
     if (edq) {
-        launch_edq_finalize(p.partials, grid, n, static_cast<collage_edq_t*>(hyper->edq_out), cs);
+        launch_edq_finalize(static_cast<EdqPartial*>(hyper->workspace), grid, n,
+                            static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
         if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
     return COLLAGE_OK;
@@ -529,7 +580,7 @@ collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const coll
         if (dispatch_step<false>(p, strategy, edq, dev.sm_count, cs, &grid) != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
     if (edq) {
-        launch_edq_finalize(p.partials, grid, plan->num_elements, static_cast<collage_edq_t*>(hyper->edq_out), cs);
+        launch_edq_finalize(p.partials, grid, plan->num_elements, static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
         if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
     return COLLAGE_OK;
@@ -544,5 +595,117 @@ collage_status_t collage_plan_destroy(collage_plan_t* plan) {
 
 uint64_t collage_plan_num_elements(const collage_plan_t* plan) { return plan ? plan->num_elements : 0; }
 uint64_t collage_plan_num_chunks(const collage_plan_t* plan) { return plan ? plan->num_chunks : 0; }
+
+// ---- state in host memory: staged step -------------------------------------------------------
+
+namespace {
+struct HostStepContext {
+    cudaStream_t in = nullptr, out = nullptr;
+    cudaEvent_t start = nullptr, loaded[2] = {nullptr, nullptr}, computed[2] = {nullptr, nullptr},
+                drained[2] = {nullptr, nullptr};
+    bool ready = false;
+};
+
+// Two copy streams and a handful of events per device, created on the first staged call.
+cudaError_t host_step_context(int device, HostStepContext** out) {
+    static HostStepContext ctx[64];
+    HostStepContext& c = ctx[device];
+    if (!c.ready) {
+        cudaError_t e;
+        if ((e = cudaStreamCreateWithFlags(&c.in, cudaStreamNonBlocking)) != cudaSuccess) return e;
+        if ((e = cudaStreamCreateWithFlags(&c.out, cudaStreamNonBlocking)) != cudaSuccess) return e;
+        cudaEvent_t* evs[] = {&c.start, &c.loaded[0], &c.loaded[1], &c.computed[0], &c.computed[1], &c.drained[0],
+                              &c.drained[1]};
+        for (cudaEvent_t* ev : evs)
+            if ((e = cudaEventCreateWithFlags(ev, cudaEventDisableTiming)) != cudaSuccess) return e;
+        c.ready = true;
+    }
+    *out = &c;
+    return cudaSuccess;
+}
+}  // namespace
+
+collage_status_t collage_adamw_step_host(void* x_hi, void* x_lo, void* m, void* v_hi, void* v_lo, const void* grad,
+                                         uint64_t n, const collage_hyper_t* hyper, uint64_t step,
+                                         collage_strategy_t strategy, void* staging_dev, size_t staging_bytes,
+                                         void* stream) {
+    if (!hyper) return COLLAGE_ERR_NULL;
+    collage_hyper_t h = *hyper;
+    void* edq_host = h.edq_out;
+    h.edq_out = nullptr;                       // workspace fields of the caller's struct are not used here
+    collage_status_t st = check_common(&h, step, strategy);
+    if (st != COLLAGE_OK) return st;
+    if (!x_hi || !m || !v_hi || !grad) return COLLAGE_ERR_NULL;
+    if ((strategy >= COLLAGE_LIGHT) != (x_lo != nullptr)) return x_lo ? COLLAGE_ERR_ARG : COLLAGE_ERR_NULL;
+    if ((strategy == COLLAGE_PLUS) != (v_lo != nullptr)) return v_lo ? COLLAGE_ERR_ARG : COLLAGE_ERR_NULL;
+    if (n > (1ull << 62)) return COLLAGE_ERR_ARG;
+    std::vector<ByteRange> ranges;
+    for (const void* q : {static_cast<const void*>(x_hi), static_cast<const void*>(x_lo), static_cast<const void*>(m),
+                          static_cast<const void*>(v_hi), static_cast<const void*>(v_lo), grad})
+        push_range(ranges, q, n);
+    if (any_overlap(ranges)) return COLLAGE_ERR_ALIAS;
+
+    // staging layout: [record 256 B][EDQ partials][2 slabs x 6 arrays x slab_elems bfloat16]
+    const size_t fixed = 256 + kWorkspaceBytes;
+    if (!staging_dev || (reinterpret_cast<uintptr_t>(staging_dev) & 255u) || staging_bytes < fixed + 2 * 6 * 2 * 16384)
+        return COLLAGE_ERR_WORKSPACE;
+    const uint64_t slab = (staging_bytes - fixed) / (2 * 6 * 2) / 16384 * 16384;
+    DeviceInfo dev;
+    st = current_device(&dev);
+    if (st != COLLAGE_OK) return st;
+    int device = 0;
+    HostStepContext* c = nullptr;
+    if (cudaGetDevice(&device) != cudaSuccess || host_step_context(device, &c) != cudaSuccess) return COLLAGE_ERR_CUDA;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    StepScalars k;
+    st = make_scalars(&h, step, &k);
+    if (st != COLLAGE_OK) return st;
+
+    char* base = static_cast<char*>(staging_dev);
+    collage_edq_t* record = reinterpret_cast<collage_edq_t*>(base);
+    EdqPartial* partials = reinterpret_cast<EdqPartial*>(base + 256);
+    uint16_t* slabs = reinterpret_cast<uint16_t*>(base + fixed);
+    auto dev_array = [&](int buf, int a) { return slabs + (static_cast<uint64_t>(buf) * 6 + a) * slab; };
+    uint16_t* host_rw[5] = {static_cast<uint16_t*>(x_hi), static_cast<uint16_t*>(x_lo), static_cast<uint16_t*>(m),
+                            static_cast<uint16_t*>(v_hi), static_cast<uint16_t*>(v_lo)};
+    const uint16_t* host_g = static_cast<const uint16_t*>(grad);
+    const bool edq = edq_host != nullptr;
+#define COLLAGE_TRY(call) do { if ((call) != cudaSuccess) return COLLAGE_ERR_CUDA; } while (0)
+
+    if (edq) COLLAGE_TRY(cudaMemsetAsync(record, 0, sizeof(collage_edq_t), cs));
+    COLLAGE_TRY(cudaEventRecord(c->start, cs));               // copies start after the caller's earlier work
+    COLLAGE_TRY(cudaStreamWaitEvent(c->in, c->start, 0));
+    const uint64_t nslabs = (n + slab - 1) / slab;
+    for (uint64_t i = 0; i < nslabs; ++i) {
+        const int b = static_cast<int>(i & 1);
+        const uint64_t off = i * slab, len = (n - off < slab) ? n - off : slab;
+        if (i >= 2) COLLAGE_TRY(cudaStreamWaitEvent(c->in, c->drained[b], 0));   // slab i-2 has left buffer b
+        for (int a = 0; a < 5; ++a)
+            if (host_rw[a])
+                COLLAGE_TRY(cudaMemcpyAsync(dev_array(b, a), host_rw[a] + off, 2 * len, cudaMemcpyHostToDevice, c->in));
+        COLLAGE_TRY(cudaMemcpyAsync(dev_array(b, 5), host_g + off, 2 * len, cudaMemcpyHostToDevice, c->in));
+        COLLAGE_TRY(cudaEventRecord(c->loaded[b], c->in));
+        COLLAGE_TRY(cudaStreamWaitEvent(cs, c->loaded[b], 0));
+        int grid = 0;
+        COLLAGE_TRY(launch_flat(dev_array(b, 0), x_lo ? dev_array(b, 1) : nullptr, dev_array(b, 2), dev_array(b, 3),
+                                v_lo ? dev_array(b, 4) : nullptr, dev_array(b, 5), len, k, strategy, edq, partials,
+                                dev.sm_count, cs, &grid));
+        if (edq) {
+            launch_edq_finalize(partials, grid, len, record, cs, true);
+            COLLAGE_TRY(cudaGetLastError());
+        }
+        COLLAGE_TRY(cudaEventRecord(c->computed[b], cs));
+        COLLAGE_TRY(cudaStreamWaitEvent(c->out, c->computed[b], 0));
+        for (int a = 0; a < 5; ++a)
+            if (host_rw[a])
+                COLLAGE_TRY(cudaMemcpyAsync(host_rw[a] + off, dev_array(b, a), 2 * len, cudaMemcpyDeviceToHost, c->out));
+        COLLAGE_TRY(cudaEventRecord(c->drained[b], c->out));
+    }
+    for (uint64_t i = (nslabs >= 2 ? nslabs - 2 : 0); i < nslabs; ++i)
+        COLLAGE_TRY(cudaStreamWaitEvent(cs, c->drained[i & 1], 0));              // results are home before `stream` goes on
+    if (edq) COLLAGE_TRY(cudaMemcpyAsync(edq_host, record, sizeof(collage_edq_t), cudaMemcpyDeviceToHost, cs));
+#undef COLLAGE_TRY
+    return COLLAGE_OK;
+}
 
 }  // extern "C"

@@ -8,11 +8,19 @@
 //   add/sub/mul/fma : the native packed instructions add/sub/mul/fma.rn.bf16x2 (sm_90+), one
 //                     rounding, subnormals kept, written as inline PTX so that nothing can be
 //                     contracted, re-associated or flushed by the compiler.
-//   div, sqrt       : no bfloat16 instruction exists.  Operands are widened to float (exact),
-//                     the IEEE-correct float result is formed (div.rn.f32 / sqrt.rn.f32), and
-//                     rounded to bfloat16 with cvt.rn.bf16x2.f32.  The float result carries 24
-//                     bits >= 2*8+2, so the second rounding cannot change the outcome for
-//                     results in the normal range.
+//   div, sqrt       : no bfloat16 instruction exists.  Operands are widened to float (exact) and
+//                     a float result q is formed that rounds (cvt.rn.bf16x2.f32) to the same
+//                     bfloat16 as the exact quotient / root:
+//                       * IEEE route: div.rn.f32 / sqrt.rn.f32.  24 bits >= 2*8+2, so the second
+//                         rounding is innocuous.
+//                       * fast route (default): a * rcp.approx.ftz(b), a * (1/b rounded to float on
+//                         the host) for the two scalar divisors, and sqrt.approx.ftz.f32.  Their relative
+//                         error is <= 2^-22, while the exact quotient of two 8-bit significands is
+//                         never an exact tie and never closer than 2^-17 (relative) to a rounding
+//                         boundary, and a square root never closer than 2^-19; so the approximation
+//                         and the exact value round alike.  The argument needs a normal-range
+//                         result: anything else (tiny, huge, Inf, NaN) takes the IEEE route; 0/b is answered directly.
+//                         collage_selftest() compares the two routes over every operand pair.
 //
 // This file is compiled only into the CUDA library; it shares nothing with the CPU oracle.
 #pragma once
@@ -58,11 +66,162 @@ __device__ __forceinline__ bf2 pack_rn(float hi, float lo) {
     return d;
 }
 
-__device__ __forceinline__ bf2 div2(bf2 a, bf2 b) {
+// two floats as one 64-bit register pair for the packed f32x2 instructions of sm_100
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 widen2(bf2 p) {      // {low half, high half} as floats (exact)
+    f32x2 d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(p << 16), "r"(p & 0xFFFF0000u));
+    return d;
+}
+__device__ __forceinline__ f32x2 splat2(float x) {
+    f32x2 d;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(d) : "f"(x));
+    return d;
+}
+__device__ __forceinline__ f32x2 mul_f32x2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 add_f32x2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 sub_f32x2(f32x2 a, f32x2 b) {
+    f32x2 d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 fma_f32x2(f32x2 a, f32x2 b, f32x2 c) {
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ float lo_of(f32x2 v) { return __uint_as_float(static_cast<uint32_t>(v)); }
+__device__ __forceinline__ float hi_of(f32x2 v) { return __uint_as_float(static_cast<uint32_t>(v >> 32)); }
+// round both floats to bfloat16 and pack (low float to the low half)
+__device__ __forceinline__ bf2 pack_rn2(f32x2 v) { return pack_rn(hi_of(v), lo_of(v)); }
+
+// IEEE routes (also the fall-back of the fast routes)
+__device__ __forceinline__ bf2 div2_ieee(bf2 a, bf2 b) {
     return pack_rn(__fdiv_rn(hi_f32(a), hi_f32(b)), __fdiv_rn(lo_f32(a), lo_f32(b)));
 }
-__device__ __forceinline__ bf2 sqrt2(bf2 a) {
+__device__ __forceinline__ bf2 sqrt2_ieee(bf2 a) {
     return pack_rn(__fsqrt_rn(hi_f32(a)), __fsqrt_rn(lo_f32(a)));
+}
+static __device__ __noinline__ float div_ieee_call(float a, float b) { return __fdiv_rn(a, b); }
+static __device__ __noinline__ float sqrt_ieee_call(float a) { return __fsqrt_rn(a); }
+
+// Quotient for operands the fast route does not cover.  A zero numerator over a normal finite
+// denominator is common (parameters that never received a gradient) and is answered directly:
+// a zero with the sign of the quotient.  Everything else goes to div.rn.f32.
+__device__ __forceinline__ float div_out_of_range(float a, float b) {
+    if (a == 0.0f && fabsf(b) >= 0x1p-126f && fabsf(b) < __uint_as_float(0x7F800000u))
+        return __uint_as_float((__float_as_uint(a) ^ __float_as_uint(b)) & 0x80000000u);
+    return div_ieee_call(a, b);
+}
+
+// single MUFU approximations; .ftz flushes subnormal inputs and outputs, which the callers below
+// either exclude or detect
+__device__ __forceinline__ float rcp_ftz(float b) {
+    float r;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(b));
+    return r;
+}
+__device__ __forceinline__ float sqrt_ftz(float a) {
+    float r;
+    asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(a));
+    return r;
+}
+
+// q is trusted only if it is a normal number with room to spare on both sides.  A subnormal
+// denominator is flushed by rcp.approx.ftz (q = Inf or NaN), a denominator above 2^126 gives a
+// flushed reciprocal (q = 0): both fail the test, as does a NaN.
+__device__ __forceinline__ bool quotient_in_fast_range(float q) {
+    return fabsf(q) >= 0x1p-125f && fabsf(q) < 0x1p127f;
+}
+
+// a (/) b, both halves, any operands
+__device__ __forceinline__ bf2 div2(bf2 a, bf2 b) {
+#ifdef COLLAGE_IEEE_DIV_SQRT
+    return div2_ieee(a, b);
+#else
+    const float a0 = lo_f32(a), a1 = hi_f32(a), b0 = lo_f32(b), b1 = hi_f32(b);
+    float q0 = __fmul_rn(a0, rcp_ftz(b0));
+    float q1 = __fmul_rn(a1, rcp_ftz(b1));
+    if (!(quotient_in_fast_range(q0) && quotient_in_fast_range(q1))) {
+        if (!quotient_in_fast_range(q0)) q0 = div_out_of_range(a0, b0);
+        if (!quotient_in_fast_range(q1)) q1 = div_out_of_range(a1, b1);
+    }
+    return pack_rn(q1, q0);
+#endif
+}
+
+// a (/) b where the caller guarantees that b is NaN, Inf, or a normal number in [2^-126, 2^126]:
+// the reciprocal is then accurate and an overflowing quotient is correctly Inf, so only a tiny
+// (possibly tied) or NaN quotient needs the IEEE route.
+__device__ __forceinline__ bf2 div2_normal_divisor(bf2 a, bf2 b) {
+#ifdef COLLAGE_IEEE_DIV_SQRT
+    return div2_ieee(a, b);
+#else
+    const float a0 = lo_f32(a), a1 = hi_f32(a), b0 = lo_f32(b), b1 = hi_f32(b);
+    float q0 = __fmul_rn(a0, rcp_ftz(b0));
+    float q1 = __fmul_rn(a1, rcp_ftz(b1));
+    if (!(fabsf(q0) >= 0x1p-125f && fabsf(q1) >= 0x1p-125f)) {
+        if (!(fabsf(q0) >= 0x1p-125f)) q0 = div_out_of_range(a0, b0);
+        if (!(fabsf(q1) >= 0x1p-125f)) q1 = div_out_of_range(a1, b1);
+    }
+    return pack_rn(q1, q0);
+#endif
+}
+
+// a (/) s for a scalar 2^-100 <= s <= 1 whose reciprocal r was rounded to float on the host.
+// No range test is needed: |a*r| >= |a|, so a quotient can only be subnormal when a is, and then
+// both the float product and the exact quotient sit on grids (2^-149 and 1/(256*2^134)) that keep
+// them on the same side of every rounding boundary; a divisor <= 1 admits no exact tie; an
+// overflowing product is the overflowing quotient; zeros, Inf and NaN pass through unchanged.
+__device__ __forceinline__ bf2 div2_by_scalar(bf2 a, float r) { return pack_rn2(mul_f32x2(widen2(a), splat2(r))); }
+
+// the same for any scalar: falls back to IEEE division when the host did not vouch (r is NaN)
+__device__ __forceinline__ bf2 div2_scalar(bf2 a, float s, float r) {
+#ifdef COLLAGE_IEEE_DIV_SQRT
+    return pack_rn(__fdiv_rn(hi_f32(a), s), __fdiv_rn(lo_f32(a), s));
+#else
+    if (r == r) return div2_by_scalar(a, r);
+    return pack_rn(__fdiv_rn(hi_f32(a), s), __fdiv_rn(lo_f32(a), s));
+#endif
+}
+
+// sqrt(a), both halves, any operand: the approximation flushes subnormal inputs, which go to sqrt.rn
+__device__ __forceinline__ bf2 sqrt2(bf2 a) {
+#ifdef COLLAGE_IEEE_DIV_SQRT
+    return sqrt2_ieee(a);
+#else
+    const float a0 = lo_f32(a), a1 = hi_f32(a);
+    float s0 = sqrt_ftz(a0), s1 = sqrt_ftz(a1);
+    if ((a0 != 0.0f && fabsf(a0) < 0x1p-126f) || (a1 != 0.0f && fabsf(a1) < 0x1p-126f)) {
+        s0 = sqrt_ieee_call(a0);
+        s1 = sqrt_ieee_call(a1);
+    }
+    return pack_rn(s1, s0);
+#endif
+}
+// all-ones in each half of the result where that half of a is < b (false for NaN)
+__device__ __forceinline__ uint32_t less_than2(bf2 a, bf2 b) {
+    uint32_t d;
+    asm("set.lt.u32.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// sqrt(a) where the caller accepts +0 for a positive subnormal input (true root < 2^-63).  A negative
+// subnormal would be flushed to -0 instead of giving NaN, so any negative lane takes the careful route.
+__device__ __forceinline__ bf2 sqrt2_flushing(bf2 a) {
+#ifdef COLLAGE_IEEE_DIV_SQRT
+    return sqrt2_ieee(a);
+#else
+    if (less_than2(a, 0u)) return sqrt2(a);
+    return pack_rn(sqrt_ftz(hi_f32(a)), sqrt_ftz(lo_f32(a)));
+#endif
 }
 
 // --------------------------------------------------------- MCF algorithms ---
@@ -127,20 +286,49 @@ struct StepScalars {
     bf2 b1, c1;        // RN(beta1), RN(1-beta1)
     bf2 b2, c2;        // RN(beta2), RN(1-beta2)
     bf2 b2h, b2l;      // beta2 as a length-2 expansion (Table 1)
-    bf2 bc1, bc2;      // RN(1-beta1^t), RN(1-beta2^t)
+    float bc1, bc2;    // RN(1-beta1^t), RN(1-beta2^t) widened to float
+    float rbc1, rbc2;  // their reciprocals rounded to float (NaN: use the IEEE route)
     bf2 neg_a;         // -RN(lr)
     bf2 lam;           // RN(weight_decay)
     bf2 eps;           // RN(eps)
-    uint32_t flags;
+    uint32_t flags;    // bit 0: epsilon under the root
+    uint32_t fast;     // host-checked: 2^-100 <= bc1, bc2 <= 1 and 2^-54 <= eps <= 2^60
 };
 
 struct ElemState {
     bf2 th, dth, m, v, dv;
 };
 
+// Algorithm 2 lines 10-12 for two parameters: the update delta from m, v (first component) and theta.
+//
+// FAST is chosen on the host when the bias corrections lie in [2^-100, 1] and 2^-54 <= eps <= 2^60
+// (every practical setting).  Then (i) the two scalar divisions need no range test, (ii) the
+// denominator is NaN, Inf or >= eps, hence a valid operand of div2_normal_divisor, and (iii) with
+// epsilon outside the root a subnormal v-hat may be flushed by the root approximation: its root is
+// below 2^-63 < ulp(eps)/2 and is absorbed by the addition of eps either way.
+template <bool FAST>
+__device__ __forceinline__ bf2 update_direction(bf2 m, bf2 v, bf2 th, const StepScalars& k) {
+    bf2 mhat, vhat, den, r;
+    if (FAST) {
+        mhat = div2_by_scalar(m, k.rbc1);
+        vhat = div2_by_scalar(v, k.rbc2);
+        if (k.flags & 1u) den = sqrt2_flushing(add2(vhat, k.eps));   // v-hat + eps >= eps: never subnormal
+        else den = add2(sqrt2_flushing(vhat), k.eps);
+        r = div2_normal_divisor(mhat, den);
+    } else {
+        mhat = div2_scalar(m, k.bc1, k.rbc1);
+        vhat = div2_scalar(v, k.bc2, k.rbc2);
+        if (k.flags & 1u) den = sqrt2(add2(vhat, k.eps));
+        else den = add2(sqrt2(vhat), k.eps);
+        r = div2(mhat, den);
+    }
+    const bf2 u = add2(r, mul2(k.lam, th));
+    return mul2(k.neg_a, u);
+}
+
 // Algorithm 2 lines 8-13 for two parameters.  STRATEGY: 0 = A, 1 = B, 2 = C.  Returns the
 // bfloat16 update of line 12; `s` is updated in place.
-template <int STRATEGY>
+template <int STRATEGY, bool FAST>
 __device__ __forceinline__ bf2 adamw_pair(ElemState& s, bf2 g, const StepScalars& k) {
     // line 8
     s.m = add2(mul2(k.b1, s.m), mul2(k.c1, g));
@@ -155,14 +343,7 @@ __device__ __forceinline__ bf2 adamw_pair(ElemState& s, bf2 g, const StepScalars
         s.v = add2(mul2(k.b2, s.v), tv);
     }
     // lines 10-12
-    const bf2 mhat = div2(s.m, k.bc1);
-    const bf2 vhat = div2(s.v, k.bc2);
-    bf2 den;
-    if (k.flags & 1u) den = sqrt2(add2(vhat, k.eps));
-    else den = add2(sqrt2(vhat), k.eps);
-    const bf2 r = div2(mhat, den);
-    const bf2 u = add2(r, mul2(k.lam, s.th));
-    const bf2 delta = mul2(k.neg_a, u);
+    const bf2 delta = update_direction<FAST>(s.m, s.v, s.th, k);
     // line 13
     if (STRATEGY == 0) {
         s.th = add2(s.th, delta);
@@ -174,31 +355,30 @@ __device__ __forceinline__ bf2 adamw_pair(ElemState& s, bf2 g, const StepScalars
     return delta;
 }
 
-// EDQ contributions of two parameters (Eq. 2-3): products in float.
+// EDQ contributions of two parameters (Eq. 2-3): differences, products and running sums in
+// float, two lanes at a time (lane = half of the bf2).
 struct EdqAcc {
-    float dot, sq;
+    f32x2 dot, sq;
     uint32_t lost;
 };
 
 template <bool HAS_LO>
 __device__ __forceinline__ void edq_pair(EdqAcc& acc, bf2 th_old, bf2 dth_old, bf2 th_new, bf2 dth_new, bf2 delta) {
-    const float d0 = lo_f32(delta), d1 = hi_f32(delta);
-    const float o0 = lo_f32(th_old), o1 = hi_f32(th_old);
-    const float n0 = lo_f32(th_new), n1 = hi_f32(th_new);
-    float e0 = __fsub_rn(n0, o0), e1 = __fsub_rn(n1, o1);
-    bool same0 = (n0 == o0), same1 = (n1 == o1);
+    const f32x2 d = widen2(delta), o = widen2(th_old), n = widen2(th_new);
+    f32x2 e = sub_f32x2(n, o);
+    bool same0 = lo_of(n) == lo_of(o), same1 = hi_of(n) == hi_of(o);
     if (HAS_LO) {
-        const float p0 = lo_f32(dth_old), p1 = hi_f32(dth_old);
-        const float q0 = lo_f32(dth_new), q1 = hi_f32(dth_new);
-        e0 = __fadd_rn(e0, __fsub_rn(q0, p0));
-        e1 = __fadd_rn(e1, __fsub_rn(q1, p1));
-        same0 = same0 && (q0 == p0);
-        same1 = same1 && (q1 == p1);
+        const f32x2 p = widen2(dth_old), q = widen2(dth_new);
+        e = add_f32x2(e, sub_f32x2(q, p));
+        same0 = same0 && lo_of(q) == lo_of(p);
+        same1 = same1 && hi_of(q) == hi_of(p);
     }
-    acc.dot = __fadd_rn(acc.dot, __fadd_rn(__fmul_rn(d0, e0), __fmul_rn(d1, e1)));
-    acc.sq = __fadd_rn(acc.sq, __fadd_rn(__fmul_rn(d0, d0), __fmul_rn(d1, d1)));
-    acc.lost += (d0 != 0.0f && same0) ? 1u : 0u;
-    acc.lost += (d1 != 0.0f && same1) ? 1u : 0u;
+    acc.dot = fma_f32x2(d, e, acc.dot);
+    acc.sq = fma_f32x2(d, d, acc.sq);
+    acc.lost += (lo_of(d) != 0.0f && same0) ? 1u : 0u;
+    acc.lost += (hi_of(d) != 0.0f && same1) ? 1u : 0u;
 }
+__device__ __forceinline__ float edq_dot(const EdqAcc& a) { return __fadd_rn(lo_of(a.dot), hi_of(a.dot)); }
+__device__ __forceinline__ float edq_sq(const EdqAcc& a) { return __fadd_rn(lo_of(a.sq), hi_of(a.sq)); }
 
 }  // namespace collage

@@ -178,3 +178,8 @@ def test_standalone_edq_matches_oracle():
         for k in ("dot", "sumsq", "edq"):
             assert abs(got[k] - want[k]) <= 1e-5 * abs(want[k])
         assert got["lost"] == want["lost"] and got["n"] == n
+
+
+def test_selftest_every_operand_pair():
+    # all 2^32 operand pairs on the device: native packed ops and the reciprocal/root shortcuts vs IEEE references
+    assert B.selftest() == dict(add=0, sub=0, mul=0, div=0, sqrt=0, scalar_div=0)

@@ -187,3 +187,96 @@ def test_wrong_device_arguments_are_rejected():
     assert err.value.status == B.ERR_ARG
     B.adamw_step(z, None, z.clone(), z.clone(), None, z.clone(), 0, h, 1, B.BF16)    # n == 0: fine, no-op
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("strategy", [0, 2])
+def test_host_resident_state_is_staged_with_identical_results(strategy):
+    # state in pinned host memory, streamed through a small device buffer so that the step takes many slabs
+    n, hyp = 300_007, W.HYPERS
+    theta = W.bits(W.flat_weights(n, 31))
+    st = oracle_state(theta, strategy)
+    host = {k: (W.from_bits(v).pin_memory() if v is not None else None) for k, v in st.items()}
+    staging = torch.empty(256 + B.workspace_bytes() + 2 * 6 * 2 * 16384 * 2 + 4096, dtype=torch.uint8, device="cuda")
+    import ctypes
+    rec = (ctypes.c_uint8 * 64)()
+    for t in (1, 2, 3):
+        g = W.bits(W.flat_grads(n, 31, t))
+        G = W.from_bits(g).pin_memory()
+        h = B.make_hyper(**hyp)
+        h.edq_out = ctypes.addressof(rec)
+        B.adamw_step_host(host["x_hi"], host["x_lo"], host["m"], host["v_hi"], host["v_lo"], G, n, h, t, strategy, staging)
+        torch.cuda.synchronize()
+        want = oracle_step(st, g, t, strategy, hyp)
+        for k in KEYS:
+            if st[k] is not None:
+                assert_same_bits(W.bits(host[k]), st[k], f"host step {t} {k}")
+        got = B.Edq.from_buffer_copy(bytes(rec)[:40])
+        edq_close(dict(dot=got.dot, sumsq=got.sumsq, edq=got.edq, lost=int(got.lost)), want)
+        assert int(got.n) == n
+    with pytest.raises(B.CollageError) as err:
+        B.adamw_step_host(host["x_hi"], host["x_lo"], host["m"], host["v_hi"], host["v_lo"], G, n, B.make_hyper(**hyp), 1,
+                          strategy, staging[:1024])
+    assert err.value.status == B.ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("eps", [0.0, 1e-40, 1e-20, 1e30])
+@pytest.mark.parametrize("flags", [0, 1])
+def test_unusual_epsilon_takes_the_guarded_arithmetic_chain(eps, flags):
+    # outside 2^-54 <= eps <= 2^60 the kernel cannot assume a normal denominator: zero and subnormal moments,
+    # zero denominators (0/0 -> NaN, x/0 -> Inf) must all come out as IEEE says
+    n, strategy = 100_000, 2
+    hyp = dict(W.HYPERS, eps=eps)
+    rng = np.random.default_rng(5)
+    theta = W.bits(W.flat_weights(n, 50))
+    st = oracle_state(theta, strategy)
+    st["v_hi"] = rng.choice(np.array([0x0000, 0x0001, 0x0040, 0x0080, 0x1000, 0x3000], np.uint16), n)
+    st["m"] = rng.choice(np.array([0x0000, 0x8000, 0x0003, 0x2000, 0xB000], np.uint16), n)
+    dev = _device_state(st)
+    for t in (1, 2):
+        g = W.bits(W.flat_grads(n, 50, t))
+        g[::3] = 0
+        G = Guarded(g)
+        B.adamw_step(_t(dev["x_hi"]), _t(dev["x_lo"]), _t(dev["m"]), _t(dev["v_hi"]), _t(dev["v_lo"]), G.t, n,
+                     B.make_hyper(**hyp, flags=flags), t, strategy)
+        torch.cuda.synchronize()
+        oracle_step(st, g, t, strategy, hyp, flags=flags)
+        _compare(dev, st, f"eps={eps} flags={flags} step {t}")
+
+
+def test_zero_and_subnormal_moments_on_the_lean_chain():
+    # default epsilon (lean chain): parameters that never saw a gradient, subnormal moments, huge moments
+    n, strategy, hyp = 100_000, 2, W.HYPERS
+    rng = np.random.default_rng(6)
+    theta = W.bits(W.flat_weights(n, 51))
+    st = oracle_state(theta, strategy)
+    st["v_hi"] = rng.choice(np.array([0x0000, 0x0001, 0x007F, 0x0080, 0x0100, 0x3000, 0x7F00, 0x7F7F], np.uint16), n)
+    st["m"] = rng.choice(np.array([0x0000, 0x8000, 0x0001, 0x8003, 0x0080, 0x2000, 0xB000, 0x7F00, 0xFF7F], np.uint16), n)
+    dev = _device_state(st)
+    e = EdqBuffers()
+    for t in (1, 2, 3):
+        g = W.bits(W.flat_grads(n, 51, t))
+        g[::2] = 0
+        G = Guarded(g)
+        B.adamw_step(_t(dev["x_hi"]), _t(dev["x_lo"]), _t(dev["m"]), _t(dev["v_hi"]), _t(dev["v_lo"]), G.t, n,
+                     e.hyper(hyp), t, strategy)
+        torch.cuda.synchronize()
+        oracle_step(st, g, t, strategy, hyp)
+        _compare(dev, st, f"lean chain step {t}")
+
+
+def test_negative_second_moment_gives_nan_not_a_flushed_zero():
+    # invalid state (v < 0, including negative subnormals) must come out NaN exactly as IEEE says
+    n, hyp = 8192, W.HYPERS
+    for strategy in (0, 2):
+        rng = np.random.default_rng(9)
+        theta = W.bits(W.flat_weights(n, 52))
+        st = oracle_state(theta, strategy)
+        st["v_hi"] = rng.choice(np.array([0x8001, 0x807F, 0x8080, 0xB000, 0x0001, 0x3000], np.uint16), n)
+        dev = _device_state(st)
+        g = np.zeros(n, np.uint16)
+        G = Guarded(g)
+        B.adamw_step(_t(dev["x_hi"]), _t(dev["x_lo"]), _t(dev["m"]), _t(dev["v_hi"]), _t(dev["v_lo"]), G.t, n,
+                     B.make_hyper(**hyp), 5, strategy)
+        torch.cuda.synchronize()
+        oracle_step(st, g, 5, strategy, hyp)
+        _compare(dev, st, f"negative v, strategy {strategy}")
