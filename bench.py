@@ -141,12 +141,14 @@ def run_collage(args):
     edq_dev = torch.zeros(64, dtype=torch.uint8, device=device)
     ws = torch.empty(B.workspace_bytes(), dtype=torch.uint8, device=device)
     edq_sums = edq_dev[:16].view(torch.float64)         # {dot, sumsq}: what ranks exchange
+    edq_lost = edq_dev[32:40].view(torch.int64)         # lost-update count
     stream = torch.cuda.current_stream()
 
     def step(t):
         B.adamw_step_multi(plan, B.make_hyper(**hyp, edq_out=edq_dev, workspace=ws), t, STRATEGY, stream)
-        if world > 1:                                   # EDQ is global: sum the two partial sums over ranks
+        if world > 1:                                   # EDQ is global: sum the partial sums over ranks
             dist.all_reduce(edq_sums)
+            dist.all_reduce(edq_lost)
 
     def barrier():
         if world > 1:
