@@ -183,6 +183,13 @@ collage_status_t collage_edq(const void* old_hi, const void* old_lo, const void*
                              const void* new_lo, const void* delta, uint64_t n, collage_edq_t* out_dev,
                              void* workspace, size_t workspace_bytes, void* stream);
 
+/* The step kernel's copy pipeline waits on shared-memory barriers with a bound of about two
+ * seconds; a wait that runs out records a code in a device word and the block leaves, so a fault
+ * can never hang the device.  This call copies that word to *out_host (0 = no fault ever seen on
+ * the current device since the last read) and clears it.  It synchronises the device: call it at
+ * checkpoints, not per step.  Errors: ERR_NULL, ERR_CUDA. */
+collage_status_t collage_pipeline_fault(uint32_t* out_host);
+
 /* Exhaustive self test of the arithmetic the kernels rely on, on the current device (Section 3.1's
  * model: one rounding to nearest-even per operation).  Compares, for EVERY pair of bfloat16 bit
  * patterns (2^32 pairs; 2^16 values for the root), the realisation used in the kernels with a

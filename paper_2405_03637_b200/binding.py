@@ -23,7 +23,7 @@ EXPORTS = (
     "collage_plan_create", "collage_adamw_step_multi", "collage_plan_destroy", "collage_plan_num_elements",
     "collage_plan_num_chunks", "collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_grow",
     "collage_scaling", "collage_mul", "collage_renormalize", "collage_rounded_op", "collage_edq",
-    "collage_selftest",
+    "collage_selftest", "collage_pipeline_fault",
 )
 
 
@@ -88,6 +88,7 @@ def lib() -> ctypes.CDLL:
         L.collage_rounded_op.argtypes = [i32, vp, vp, vp, vp, u64, vp]
         L.collage_edq.argtypes = [vp, vp, vp, vp, vp, u64, vp, vp, ctypes.c_size_t, vp]
         L.collage_selftest.argtypes = [ctypes.POINTER(ctypes.c_uint64), vp]
+        L.collage_pipeline_fault.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
         _lib = L
     return _lib
 
@@ -209,6 +210,12 @@ def selftest(stream=None) -> dict:
     out = (ctypes.c_uint64 * 6)()
     _check(lib().collage_selftest(out, _ptr(stream)), "collage_selftest")
     return dict(zip(("add", "sub", "mul", "div", "sqrt", "scalar_div"), (int(v) for v in out)))
+
+
+def pipeline_fault() -> int:
+    out = ctypes.c_uint32(0)
+    _check(lib().collage_pipeline_fault(ctypes.byref(out)), "collage_pipeline_fault")
+    return int(out.value)
 
 
 def read_edq(edq_dev) -> dict:

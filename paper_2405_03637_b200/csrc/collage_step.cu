@@ -12,8 +12,27 @@
 
 namespace collage {
 
-// Launch geometry of the step kernel (measured on B200: 128 threads x 6 resident blocks per SM,
-// one 8-element vector per thread in flight, 80 registers, was the fastest of the shapes tried).
+// Default data movement: the bulk-copy pipeline of step_pipeline.cuh.  Measured on B200 (2^30
+// parameters, Collage-plus with EDQ, median of 80 launches): 512 consumer threads + one producer warp,
+// one block per SM, three stages of 4096-element tiles reached 6.47 TB/s; the register-staged kernel
+// below (-DCOLLAGE_PLAIN_KERNEL) 6.07 TB/s; smaller tiles, more stages or two blocks per SM were slower.
+#ifndef COLLAGE_PLAIN_KERNEL
+#define COLLAGE_USE_PIPELINE 1
+#endif
+#ifndef COLLAGE_PIPE_CONSUMERS
+#define COLLAGE_PIPE_CONSUMERS 512
+#endif
+#ifndef COLLAGE_PIPE_VPT
+#define COLLAGE_PIPE_VPT 1
+#endif
+#ifndef COLLAGE_PIPE_STAGES
+#define COLLAGE_PIPE_STAGES 3
+#endif
+#ifndef COLLAGE_PIPE_MINBLOCKS
+#define COLLAGE_PIPE_MINBLOCKS 1
+#endif
+// Launch geometry of the register-staged kernel (128 threads x 6 resident blocks per SM, one
+// 8-element vector per thread in flight, 80 registers, was the fastest of the shapes tried).
 #ifndef COLLAGE_THREADS
 #define COLLAGE_THREADS 128
 #endif
@@ -25,6 +44,11 @@ namespace collage {
 #endif
 constexpr int kThreads = COLLAGE_THREADS;
 constexpr uint32_t kDefaultChunk = 16384;
+#ifdef COLLAGE_USE_PIPELINE
+constexpr uint32_t kFlatChunk = COLLAGE_PIPE_CONSUMERS * 8 * COLLAGE_PIPE_VPT * 4;   // four tiles
+#else
+constexpr uint32_t kFlatChunk = kDefaultChunk;
+#endif
 
 struct TensorRec {
     uint16_t* x_hi;
@@ -54,11 +78,37 @@ struct StepParams {
 };
 
 // ---- 16-byte streaming accesses (each byte is touched once: do not keep it in L1) ----------
+#ifndef COLLAGE_LD_POLICY
+#define COLLAGE_LD_POLICY 0
+#endif
+#ifndef COLLAGE_ST_POLICY
+#define COLLAGE_ST_POLICY 0
+#endif
 __device__ __forceinline__ uint4 ld_stream(const uint16_t* p) {
+#if COLLAGE_LD_POLICY == 0
     return __ldcs(reinterpret_cast<const uint4*>(p));
+#elif COLLAGE_LD_POLICY == 1
+    return *reinterpret_cast<const uint4*>(p);
+#elif COLLAGE_LD_POLICY == 2
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+#else
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.L2::evict_first.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+#endif
 }
 __device__ __forceinline__ void st_stream(uint16_t* p, const uint4& v) {
+#if COLLAGE_ST_POLICY == 0
     __stcs(reinterpret_cast<uint4*>(p), v);
+#elif COLLAGE_ST_POLICY == 1
+    *reinterpret_cast<uint4*>(p) = v;
+#elif COLLAGE_ST_POLICY == 2
+    __stwt(reinterpret_cast<uint4*>(p), v);
+#else
+    asm volatile("st.global.L1::no_allocate.L2::evict_first.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+#endif
 }
 
 // element-wise gather/scatter of up to 8 bfloat16 values into / out of four packed registers
@@ -91,6 +141,10 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
     uint32_t* dv = reinterpret_cast<uint32_t*>(&s.dv);
     const uint32_t* g = reinterpret_cast<const uint32_t*>(&s.g);
     EdqAcc acc = {0ull, 0ull, 0u};
+#ifdef COLLAGE_NULL_COMPUTE
+    th[0] ^= g[0] & 1u;   // data-movement experiment only: no arithmetic
+    return;
+#endif
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         ElemState e;
@@ -159,6 +213,10 @@ __device__ __forceinline__ void store_elems(const Vec& s, const TensorRec& t, ui
     if (STRATEGY >= 1) st_elems(t.x_lo + off, s.dth, count);
     if (STRATEGY == 2) st_elems(t.v_lo + off, s.dv, count);
 }
+
+}  // namespace collage
+#include "step_pipeline.cuh"
+namespace collage {
 
 template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, int UNROLL>
 __global__ void __launch_bounds__(kThreads, COLLAGE_MINBLOCKS) adamw_step_kernel(const __grid_constant__ StepParams p) {
@@ -326,20 +384,38 @@ static collage_status_t make_scalars(const collage_hyper_t* hyper, uint64_t step
 
 template <int STRATEGY, bool EDQ, bool FLAT, bool FAST>
 static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t stream, int* grid_out) {
-    constexpr int UNROLL = COLLAGE_UNROLL;
-    auto kernel = adamw_step_kernel<STRATEGY, EDQ, FLAT, FAST, UNROLL>;
+#ifdef COLLAGE_USE_PIPELINE
+    constexpr int CONSUMERS = COLLAGE_PIPE_CONSUMERS, VPT = COLLAGE_PIPE_VPT, STAGES = COLLAGE_PIPE_STAGES;
+    auto kernel = adamw_step_pipeline_kernel<STRATEGY, EDQ, FLAT, FAST, CONSUMERS, VPT, STAGES>;
+    constexpr size_t smem = sizeof(PipeSmem<CONSUMERS, VPT, STAGES, STRATEGY>) + 128;
+    constexpr int threads = CONSUMERS + 32;
     static int blocks_per_sm = 0;   // per instantiation
     if (blocks_per_sm == 0) {
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+        if (e != cudaSuccess) return e;
         int b = 0;
-        const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, kThreads, 0);
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, threads, smem);
         if (e != cudaSuccess) return e;
         blocks_per_sm = b > 0 ? b : 1;
     }
+#else
+    constexpr int UNROLL = COLLAGE_UNROLL;
+    auto kernel = adamw_step_kernel<STRATEGY, EDQ, FLAT, FAST, UNROLL>;
+    constexpr size_t smem = 0;
+    constexpr int threads = kThreads;
+    static int blocks_per_sm = 0;   // per instantiation
+    if (blocks_per_sm == 0) {
+        int b = 0;
+        const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, threads, 0);
+        if (e != cudaSuccess) return e;
+        blocks_per_sm = b > 0 ? b : 1;
+    }
+#endif
     uint64_t grid = static_cast<uint64_t>(sm_count) * blocks_per_sm;
     if (grid > p.num_chunks) grid = p.num_chunks;
     if (grid > static_cast<uint64_t>(kMaxGrid)) grid = kMaxGrid;
     *grid_out = static_cast<int>(grid);
-    kernel<<<static_cast<unsigned>(grid), kThreads, 0, stream>>>(p);
+    kernel<<<static_cast<unsigned>(grid), threads, smem, stream>>>(p);
     return cudaGetLastError();
 }
 
@@ -381,8 +457,8 @@ static cudaError_t launch_flat(void* x_hi, void* x_lo, void* m, void* v_hi, void
     p.flat.n = n;
     p.flat.aligned = aligned16(x_hi) && aligned16(x_lo) && aligned16(m) && aligned16(v_hi) && aligned16(v_lo) &&
                      aligned16(grad);
-    p.chunk_elems = kDefaultChunk;
-    p.num_chunks = (n + kDefaultChunk - 1) / kDefaultChunk;
+    p.chunk_elems = kFlatChunk;
+    p.num_chunks = (n + kFlatChunk - 1) / kFlatChunk;
     p.partials = partials;
     return dispatch_step<true>(p, strategy, edq, sm_count, stream, grid_out);
 }
@@ -595,6 +671,15 @@ collage_status_t collage_plan_destroy(collage_plan_t* plan) {
 
 uint64_t collage_plan_num_elements(const collage_plan_t* plan) { return plan ? plan->num_elements : 0; }
 uint64_t collage_plan_num_chunks(const collage_plan_t* plan) { return plan ? plan->num_chunks : 0; }
+
+collage_status_t collage_pipeline_fault(uint32_t* out_host) {
+    if (!out_host) return COLLAGE_ERR_NULL;
+    unsigned int v = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&v, g_pipeline_fault, sizeof v) != cudaSuccess) return COLLAGE_ERR_CUDA;
+    if (v && cudaMemcpyToSymbol(g_pipeline_fault, &zero, sizeof zero) != cudaSuccess) return COLLAGE_ERR_CUDA;
+    *out_host = v;
+    return COLLAGE_OK;
+}
 
 // ---- state in host memory: staged step -------------------------------------------------------
 

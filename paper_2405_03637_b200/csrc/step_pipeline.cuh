@@ -1,0 +1,303 @@
+// Bulk-copy pipelined variant of the fused AdamW step.
+//
+// Same arithmetic and same chunk walk as adamw_step_kernel, different data movement: one
+// producer thread per block moves whole tiles (kTile elements of every state array) between
+// global and shared memory with the bulk asynchronous copy engine (cp.async.bulk, completion on
+// an mbarrier), kStages tiles deep, while the consumer warps compute out of shared memory and
+// write their results back into the same shared slots, from where the producer bulk-stores them.
+// Bytes in flight per SM no longer depend on registers or on how long the arithmetic takes.
+//
+//   full[s]  : producer -> consumers, "tile in stage s has landed" (1 arrival + transaction bytes)
+//   done[s]  : consumers -> producer, "stage s is computed and written back" (one arrival per warp)
+//
+// Tiles that cannot be bulk-copied (tensor not 16-byte aligned, or the ragged last tile of a
+// tensor) flow through the same barriers but are processed straight from global memory.
+// Every wait is bounded: after ~2 s a thread records a fault in g_pipeline_fault and leaves.
+#pragma once
+#include "mcf_device.cuh"
+
+namespace collage {
+
+__device__ unsigned int g_pipeline_fault = 0;   // 0 = none; else 1 + index of the wait that gave up
+
+namespace pipe {
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after ~4e9 cycles (about two seconds), records which wait failed.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int who) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (clock64() - t0 > 4000000000LL) {
+            atomicCAS(&g_pipeline_fault, 0u, who + 1u);
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_addr(smem_dst)),
+                 "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gmem_dst), "r"(smem_addr(smem_src)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+}  // namespace pipe
+
+// Number of state arrays read / written per option
+template <int STRATEGY>
+struct ArrayCount {
+    static constexpr int kIn = 4 + (STRATEGY >= 1 ? 1 : 0) + (STRATEGY == 2 ? 1 : 0);
+    static constexpr int kOut = kIn - 1;   // everything but the gradient
+};
+
+// order of the arrays inside a stage: th, m, v, [dth], [dv], g  (outputs first, gradient last)
+template <int STRATEGY>
+__device__ __forceinline__ void tile_pointers(const TensorRec& t, uint64_t off, uint16_t* (&out)[5], const uint16_t*& g) {
+    int a = 0;
+    out[a++] = t.x_hi + off;
+    out[a++] = t.m + off;
+    out[a++] = t.v_hi + off;
+    if (STRATEGY >= 1) out[a++] = t.x_lo + off;
+    if (STRATEGY == 2) out[a++] = t.v_lo + off;
+    g = t.grad + off;
+}
+
+template <int CONSUMERS, int VPT, int STAGES, int STRATEGY>
+struct PipeSmem {
+    static constexpr int kTile = CONSUMERS * 8 * VPT;
+    alignas(128) uint16_t data[STAGES][ArrayCount<STRATEGY>::kIn][kTile];
+    alignas(8) uint64_t full[STAGES];
+    alignas(8) uint64_t done[STAGES];
+    double red_dot[CONSUMERS / 32], red_sq[CONSUMERS / 32];
+    unsigned long long red_lost[CONSUMERS / 32];
+};
+
+template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, int CONSUMERS, int VPT, int STAGES>
+__global__ void __launch_bounds__(CONSUMERS + 32, COLLAGE_PIPE_MINBLOCKS)
+adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
+    constexpr int kTile = CONSUMERS * 8 * VPT;
+    constexpr int NIN = ArrayCount<STRATEGY>::kIn, NOUT = ArrayCount<STRATEGY>::kOut;
+    constexpr int kWarps = CONSUMERS / 32;
+    extern __shared__ unsigned char smem_raw[];
+    using Smem = PipeSmem<CONSUMERS, VPT, STAGES, STRATEGY>;
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
+
+    const bool is_producer = threadIdx.x >= CONSUMERS;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int s = 0; s < STAGES; ++s) {
+            pipe::mbar_init(&sm.full[s], 1);
+            pipe::mbar_init(&sm.done[s], kWarps);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    double dot = 0.0, sq = 0.0;
+    uint32_t lost = 0;
+    const StepScalars& k = p.k;
+    uint32_t it = 0;          // running tile number of this block; both roles count the same sequence
+    bool alive = true;
+
+    if (is_producer) {
+        if (threadIdx.x == CONSUMERS) {
+            // what sits in each stage, so that it can be stored out once the consumers are done with it
+            uint16_t* held_out[STAGES][5];
+            uint32_t held_bytes[STAGES];
+#pragma unroll
+            for (int s = 0; s < STAGES; ++s) held_bytes[s] = 0;
+
+            for (uint64_t c = blockIdx.x; c < p.num_chunks && alive; c += gridDim.x) {
+                TensorRec t;
+                uint64_t start;
+                if (FLAT) {
+                    t = p.flat;
+                    start = c * p.chunk_elems;
+                } else {
+                    const ChunkRec cr = p.chunks[c];
+                    t = p.tensors[cr.tensor];
+                    start = static_cast<uint64_t>(cr.index) * p.chunk_elems;
+                }
+                const uint64_t left = t.n - start;
+                const uint32_t len = left < p.chunk_elems ? static_cast<uint32_t>(left) : p.chunk_elems;
+                for (uint32_t off = 0; off < len && alive; off += kTile, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t use = it / STAGES;
+                    if (use > 0) {   // the stage still holds tile it - STAGES: wait for it, send it home
+                        alive = pipe::mbar_wait(&sm.done[s], (use - 1) & 1u, 10u + s);
+                        if (!alive) break;
+                        if (held_bytes[s]) {
+#pragma unroll
+                            for (int a = 0; a < NOUT; ++a) pipe::bulk_store(held_out[s][a], sm.data[s][a], held_bytes[s]);
+                            pipe::bulk_commit();
+                            pipe::bulk_wait_read_all();   // the stage may be overwritten once it has been read out
+                        }
+                    }
+                    const uint32_t tl = (len - off) < static_cast<uint32_t>(kTile) ? (len - off) : kTile;
+                    const bool bulk = t.aligned && tl == static_cast<uint32_t>(kTile);
+                    if (bulk) {
+                        const uint16_t* g;
+                        tile_pointers<STRATEGY>(t, start + off, held_out[s], g);
+                        held_bytes[s] = kTile * 2;
+                        pipe::mbar_arrive_expect_tx(&sm.full[s], NIN * kTile * 2);
+#pragma unroll
+                        for (int a = 0; a < NOUT; ++a) pipe::bulk_load(sm.data[s][a], held_out[s][a], kTile * 2, &sm.full[s]);
+                        pipe::bulk_load(sm.data[s][NOUT], g, kTile * 2, &sm.full[s]);
+                    } else {
+                        held_bytes[s] = 0;
+                        pipe::mbar_arrive(&sm.full[s]);
+                    }
+                }
+            }
+            // drain: the last min(it, STAGES) tiles are still in their stages
+            const uint32_t tail = it < static_cast<uint32_t>(STAGES) ? it : STAGES;
+            for (uint32_t j = it - tail; j < it && alive; ++j) {
+                const int s = j % STAGES;
+                alive = pipe::mbar_wait(&sm.done[s], (j / STAGES) & 1u, 20u + s);
+                if (!alive) break;
+                if (held_bytes[s]) {
+#pragma unroll
+                    for (int a = 0; a < NOUT; ++a) pipe::bulk_store(held_out[s][a], sm.data[s][a], held_bytes[s]);
+                    pipe::bulk_commit();
+                }
+            }
+            if (!alive) {
+                // a wait gave up: loads already issued still land in shared memory; let them finish
+                for (int s = 0; s < STAGES; ++s) {
+                    const uint32_t armed = (it > static_cast<uint32_t>(s)) ? (it - 1 - s) / STAGES : 0;
+                    if (it > static_cast<uint32_t>(s)) pipe::mbar_wait(&sm.full[s], armed & 1u, 30u + s);
+                }
+            }
+            pipe::bulk_wait_all();
+        }
+    } else {
+        const int lane = threadIdx.x & 31;
+        for (uint64_t c = blockIdx.x; c < p.num_chunks && alive; c += gridDim.x) {
+            TensorRec t;
+            uint64_t start;
+            if (FLAT) {
+                t = p.flat;
+                start = c * p.chunk_elems;
+            } else {
+                const ChunkRec cr = p.chunks[c];
+                t = p.tensors[cr.tensor];
+                start = static_cast<uint64_t>(cr.index) * p.chunk_elems;
+            }
+            const uint64_t left = t.n - start;
+            const uint32_t len = left < p.chunk_elems ? static_cast<uint32_t>(left) : p.chunk_elems;
+            for (uint32_t off = 0; off < len; off += kTile, ++it) {
+                const int s = it % STAGES;
+                alive = pipe::mbar_wait(&sm.full[s], (it / STAGES) & 1u, 40u + s);
+                if (!alive) break;
+                const uint32_t tl = (len - off) < static_cast<uint32_t>(kTile) ? (len - off) : kTile;
+                if (t.aligned && tl == static_cast<uint32_t>(kTile)) {
+#pragma unroll
+                    for (int j = 0; j < VPT; ++j) {
+                        Vec v;
+                        const int e = (j * CONSUMERS + threadIdx.x) * 8;
+                        int a = 0;
+                        v.th = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
+                        v.m = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
+                        v.v = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
+                        if (STRATEGY >= 1) v.dth = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
+                        if (STRATEGY == 2) v.dv = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
+                        v.g = *reinterpret_cast<const uint4*>(&sm.data[s][a][e]);
+                        compute_vec<STRATEGY, EDQ, FAST>(v, k, 8, dot, sq, lost);
+                        a = 0;
+                        *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.th;
+                        *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.m;
+                        *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.v;
+                        if (STRATEGY >= 1) *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.dth;
+                        if (STRATEGY == 2) *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.dv;
+                    }
+                    pipe::fence_async_smem();      // shared-memory writes must be visible to the bulk store
+                } else {
+                    // straight from global memory: vectors where the tensor allows, elements otherwise
+                    const uint32_t nvec = tl >> 3;
+                    const int rem = static_cast<int>(tl & 7u);
+                    const uint64_t base = start + off;
+                    for (uint32_t i = threadIdx.x; i < nvec; i += CONSUMERS) {
+                        Vec v;
+                        if (t.aligned) load_vec<STRATEGY>(v, t, base + 8ull * i);
+                        else load_elems<STRATEGY>(v, t, base + 8ull * i, 8);
+                        compute_vec<STRATEGY, EDQ, FAST>(v, k, 8, dot, sq, lost);
+                        if (t.aligned) store_vec<STRATEGY>(v, t, base + 8ull * i);
+                        else store_elems<STRATEGY>(v, t, base + 8ull * i, 8);
+                    }
+                    if (rem && threadIdx.x == (nvec % CONSUMERS)) {
+                        Vec v;
+                        load_elems<STRATEGY>(v, t, base + 8ull * nvec, rem);
+                        compute_vec<STRATEGY, EDQ, FAST>(v, k, rem, dot, sq, lost);
+                        store_elems<STRATEGY>(v, t, base + 8ull * nvec, rem);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) pipe::mbar_arrive(&sm.done[s]);
+            }
+        }
+    }
+
+    if (EDQ) {
+        unsigned long long lost64 = lost;
+        if (!is_producer) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                dot += __shfl_down_sync(0xFFFFFFFFu, dot, o);
+                sq += __shfl_down_sync(0xFFFFFFFFu, sq, o);
+                lost64 += __shfl_down_sync(0xFFFFFFFFu, lost64, o);
+            }
+            if ((threadIdx.x & 31) == 0) {
+                sm.red_dot[threadIdx.x >> 5] = dot;
+                sm.red_sq[threadIdx.x >> 5] = sq;
+                sm.red_lost[threadIdx.x >> 5] = lost64;
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            double d = 0.0, q = 0.0;
+            unsigned long long l = 0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                d += sm.red_dot[w];
+                q += sm.red_sq[w];
+                l += sm.red_lost[w];
+            }
+            p.partials[blockIdx.x] = EdqPartial{d, q, l, 0ull};
+        }
+    }
+}
+
+}  // namespace collage
