@@ -43,7 +43,8 @@ typedef enum {
     COLLAGE_ERR_ALIAS = 3,      /* two tensors of one call overlap                              */
     COLLAGE_ERR_ARCH = 4,       /* current device is not sm_100                                 */
     COLLAGE_ERR_CUDA = 5,       /* a CUDA runtime call or launch failed                         */
-    COLLAGE_ERR_WORKSPACE = 6   /* workspace missing or smaller than collage_workspace_bytes()  */
+    COLLAGE_ERR_WORKSPACE = 6,  /* workspace missing or smaller than collage_workspace_bytes()  */
+    COLLAGE_ERR_LIMIT = 7       /* size beyond the fixed capacity of an entry point             */
 } collage_status_t;
 
 /* Precision options of Table 2. */
@@ -182,6 +183,31 @@ collage_status_t collage_rounded_op(int op, const void* a, const void* b, const 
 collage_status_t collage_edq(const void* old_hi, const void* old_lo, const void* new_hi,
                              const void* new_lo, const void* delta, uint64_t n, collage_edq_t* out_dev,
                              void* workspace, size_t workspace_bytes, void* stream);
+
+/* EDQ for callers that cannot allocate device memory (the paper has no counterpart; this is an
+ * interface convenience, the computation is collage_edq's).  Some callers own no allocator they
+ * may call at this point: a training process that has handed every byte of the GPU to a memory
+ * pool and forbids raw cudaMalloc inside the step (it can fail, and it synchronises the device),
+ * a plugin running inside someone else's framework without access to its allocator, or code in a
+ * latency-critical region.  For them the scratch that collage_edq takes as `workspace` is built
+ * into the library: a fixed 64 KiB array in device memory (2048 partial sums), which every GPU
+ * that loads the library holds until the process exits.  Arguments are those of collage_edq
+ * without workspace; `out_dev` is still the caller's DEVICE collage_edq_t.
+ *   - Capacity: one partial sum per 2^21 elements, so n <= 2^32; a larger n is rejected with
+ *     COLLAGE_ERR_LIMIT and nothing is launched.
+ *   - The call itself allocates nothing and frees nothing.  The first call on each device looks up
+ *     the array's device address (cudaGetSymbolAddress, with that device current); make that first
+ *     call before any stream capture begins.
+ *   - All calls on a device share the one array.  Each call overwrites every slot it later reads,
+ *     so nothing needs clearing between calls; but two calls whose kernels overlap on the GPU
+ *     (different streams, no ordering) race on it.  Order them, or use collage_edq with separate
+ *     workspaces.
+ *   - The sums are grouped per fixed 2^21-element segment, not per launch geometry, so they can
+ *     differ from collage_edq's in the last bits (same tolerance as against the CPU oracle).
+ * Errors: ERR_NULL, ERR_LIMIT, ERR_ARCH, ERR_CUDA. */
+collage_status_t collage_edq_static(const void* old_hi, const void* old_lo, const void* new_hi,
+                                    const void* new_lo, const void* delta, uint64_t n,
+                                    collage_edq_t* out_dev, void* stream);
 
 /* The step kernel's copy pipeline waits on shared-memory barriers with a bound of about two
  * seconds; a wait that runs out records a code in a device word and the block leaves, so a fault

@@ -11,7 +11,7 @@ from pathlib import Path
 
 _LIB_PATH = Path(__file__).resolve().parent / "libcollage_b200.so"
 
-OK, ERR_NULL, ERR_ARG, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_WORKSPACE = range(7)
+OK, ERR_NULL, ERR_ARG, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_WORKSPACE, ERR_LIMIT = range(8)
 BF16, LIGHT, PLUS = 0, 1, 2
 FLAG_EPS_INSIDE_SQRT = 1
 OP_ADD, OP_SUB, OP_MUL, OP_DIV, OP_SQRT, OP_FMA = range(6)
@@ -23,7 +23,7 @@ EXPORTS = (
     "collage_plan_create", "collage_adamw_step_multi", "collage_plan_destroy", "collage_plan_num_elements",
     "collage_plan_num_chunks", "collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_grow",
     "collage_scaling", "collage_mul", "collage_renormalize", "collage_rounded_op", "collage_edq",
-    "collage_selftest", "collage_pipeline_fault",
+    "collage_selftest", "collage_pipeline_fault", "collage_edq_static",
 )
 
 
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.collage_mul.argtypes = [vp, vp, vp, vp, vp, vp, u64, vp]
         L.collage_rounded_op.argtypes = [i32, vp, vp, vp, vp, u64, vp]
         L.collage_edq.argtypes = [vp, vp, vp, vp, vp, u64, vp, vp, ctypes.c_size_t, vp]
+        L.collage_edq_static.argtypes = [vp, vp, vp, vp, vp, u64, vp, vp]
         L.collage_selftest.argtypes = [ctypes.POINTER(ctypes.c_uint64), vp]
         L.collage_pipeline_fault.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
         _lib = L
@@ -204,6 +205,12 @@ def edq(old_hi, old_lo, new_hi, new_lo, delta, n, out_dev, workspace, stream=Non
     ws_bytes = workspace.numel() * workspace.element_size()
     _check(lib().collage_edq(_ptr(old_hi), _ptr(old_lo), _ptr(new_hi), _ptr(new_lo), _ptr(delta), n, _ptr(out_dev),
                              _ptr(workspace), ws_bytes, _ptr(stream)), "collage_edq")
+
+
+def edq_static(old_hi, old_lo, new_hi, new_lo, delta, n, out_dev, stream=None):
+    """EDQ with the library's built-in scratch: for callers that cannot allocate a workspace (n <= 2^32)."""
+    _check(lib().collage_edq_static(_ptr(old_hi), _ptr(old_lo), _ptr(new_hi), _ptr(new_lo), _ptr(delta), n,
+                                    _ptr(out_dev), _ptr(stream)), "collage_edq_static")
 
 
 def selftest(stream=None) -> dict:

@@ -502,6 +502,7 @@ const char* collage_status_string(collage_status_t status) {
         case COLLAGE_ERR_ARCH: return "current device is not compute capability 10.x (sm_100a only, no fallback)";
         case COLLAGE_ERR_CUDA: return "CUDA runtime error";
         case COLLAGE_ERR_WORKSPACE: return "EDQ workspace missing, misaligned or too small";
+        case COLLAGE_ERR_LIMIT: return "size beyond the fixed capacity of this entry point";
     }
     return "unknown status";
 }
