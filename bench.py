@@ -27,6 +27,10 @@ UNIT = "params/s"
 BYTES_PER_PARAM = {0: 14, 1: 18, 2: 22}      # algorithmic HBM bytes per parameter per step (A, B, C)
 STRATEGY = 2                                  # Collage-plus
 WORKLOAD = "llama7b_shaped_291_tensors_collage_plus_with_edq"
+# DRAM bytes per parameter of the step kernel from one ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum = 3.146 GB + 2.565 GB on the 262,148,096-parameter case, summary under
+# profiles/); every byte is touched once, so traffic scales with the parameter count.
+NCU_TRAFFIC_BYTES_PER_PARAM = (3.146196e9 + 2.565302e9) / 262_148_096
 
 
 def measured_hbm_peak():
@@ -194,8 +198,9 @@ def run_collage(args):
                    "parallelism": f"dp{world} (each rank owns a full 7B-shaped shard; EDQ sums all-reduced)"},
         "gpu_launches": 2 * args.steps,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": args.traffic_gb, "peak_source": peak_src, "frac_of_nominal_8TBps": achieved / 8000.0,
-                     "kernel": "adamw_step_kernel<C, EDQ, multi>", "kernel_ms": kernel_ms},
+                     "traffic": NCU_TRAFFIC_BYTES_PER_PARAM * n / 1e9, "traffic_unit": "GB per launch (ncu, scaled by parameters)",
+                     "algorithmic": n * BYTES_PER_PARAM[STRATEGY] / 1e9, "peak_source": peak_src, "frac_of_nominal_8TBps": achieved / 8000.0,
+                     "kernel": "adamw_step_pipeline_kernel<C, EDQ, multi-tensor>", "kernel_ms": kernel_ms},
         "clocks": clocks.summary(),
         "edq": edq["edq"],
     }
@@ -316,8 +321,6 @@ def main():
     ap.add_argument("--layers", type=int, default=32, help="transformer layers of the 7B-shaped set (32 = full)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--skip-extras", action="store_true", help="no e2e and no CPU baseline (profiling runs)")
-    ap.add_argument("--traffic-gb", type=float, default=None,
-                    help="per-launch DRAM traffic (GB) from the ncu capture recorded under profiles/")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -2,11 +2,16 @@
 // streams every state array exactly once, plus the entry points that launch it.
 //
 // Work is cut into chunks of `chunk_elems` consecutive elements of one tensor.  Thread block b
-// takes chunks b, b + grid, b + 2*grid, ...  Inside a chunk each thread owns 8 consecutive
-// elements (one 16-byte vector per state array) at a time.  Tensors whose pointers are not all
-// 16-byte aligned, and the last (<8) elements of a tensor, go through an element-wise path that
-// feeds the same arithmetic.  EDQ sums: float within a vector, double per thread, fixed-order
-// tree per block, one partial per block, summed by a one-block finalize kernel.
+// takes chunks b, b + grid, b + 2*grid, ...  Two kernels walk the chunks the same way:
+//   * step_pipeline.cuh (default): tiles are moved between global and shared memory by the bulk
+//     asynchronous copy engine, the threads compute out of shared memory;
+//   * adamw_step_kernel below (-DCOLLAGE_PLAIN_KERNEL): each thread loads 16-byte vectors into
+//     registers, computes, stores.
+// In both, a thread owns 8 consecutive elements (one 16-byte vector per state array) at a time;
+// tensors whose pointers are not all 16-byte aligned, and the last (<8) elements of a tensor, go
+// through an element-wise path that feeds the same arithmetic.  EDQ sums: float within a vector,
+// double per thread, fixed-order tree per block, one partial per block, summed by a one-block
+// finalize kernel.
 #include "host_common.cuh"
 #include "mcf_device.cuh"
 
