@@ -1,0 +1,191 @@
+"""GPU parity on the benchmark's own configurations, including the full-size LLaMA-7B-shaped launch.
+
+Full-size arrays are far beyond what the oracle can step in seconds, so the large cases compare
+sampled windows (every element of a window bit for bit; elements are independent, so a window is a
+complete check of the elements in it) and the small cases compare whole arrays.
+"""
+import numpy as np
+import pytest
+import torch
+
+import bench
+import oracle
+from gpu_util import EdqBuffers, assert_same_bits, edq_close, oracle_step
+from paper_2405_03637_b200 import binding as B
+from paper_2405_03637_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+KEYS = ("x_hi", "x_lo", "m", "v_hi", "v_lo")
+
+
+def _windows(n, rng, width, count):
+    """Sample windows of one tensor: its first and last `width` elements and `count` random ones."""
+    if n <= 2 * width:
+        return [(0, n)]
+    wins = [(0, width), (n - width, n)]
+    for _ in range(count):
+        lo = int(rng.integers(0, n - width))
+        wins.append((lo, lo + width))
+    return wins
+
+
+def _gather(t, wins):
+    return np.concatenate([W.bits(t[lo:hi]) for lo, hi in wins])
+
+
+def test_llama7b_full_size_launch_sampled_parity():
+    # the exact launch bench.py times: 291 tensors, 6,738,415,616 parameters, Collage-plus with EDQ
+    dev = torch.device("cuda")
+    arrays, rows, n = bench.build_llama7b_state(torch, W, dev, seed=3, layers=32)
+    assert n == 6_738_415_616 and len(rows) == 291
+    plan = B.plan_create(rows)
+    assert B.plan_num_elements(plan) == n
+    e = EdqBuffers()
+    rng = np.random.default_rng(0)
+    samples = []                                   # (row index, windows, oracle state dict, gradient bits)
+    for i, row in enumerate(rows):
+        wins = _windows(row[6], rng, 4096, 6)
+        st = {k: _gather(row[j], wins) for j, k in enumerate(KEYS)}
+        samples.append((i, wins, st, _gather(row[5], wins)))
+    total = sum(sum(hi - lo for lo, hi in wins) for _, wins, _, _ in samples)
+    assert total > 6_000_000
+    hyp = W.HYPERS
+    for t in (1, 2):
+        B.adamw_step_multi(plan, e.hyper(hyp), t, B.PLUS)
+        torch.cuda.synchronize()
+        for i, wins, st, g in samples:
+            oracle_step(st, g, t, 2, hyp)
+            for j, k in enumerate(KEYS):
+                assert_same_bits(_gather(rows[i][j], wins), st[k], f"step {t} tensor {i} {k}")
+        got = e.read()
+        assert got["n"] == n and 0 <= got["lost"] <= n
+        assert np.isfinite(got["edq"]) and got["edq"] > 0 and got["sumsq"] > 0
+        assert abs(got["edq"]) <= np.sqrt(got["sumsq"]) * 1.5          # projection of a nearby vector
+    assert B.pipeline_fault() == 0
+    B.plan_destroy(plan)
+    del arrays, rows
+    torch.cuda.empty_cache()
+
+
+def test_llama7b_layout_one_layer_whole_arrays_and_edq():
+    # the same layout with one transformer layer (464 M parameters): every element and the global EDQ
+    dev = torch.device("cuda")
+    arrays, rows, n = bench.build_llama7b_state(torch, W, dev, seed=3, layers=1)
+    plan = B.plan_create(rows)
+    e = EdqBuffers()
+    st = {k: W.bits(arrays[k]) for k in KEYS}
+    g = W.bits(arrays["grad"])
+    B.adamw_step_multi(plan, e.hyper(W.HYPERS), 1, B.PLUS)
+    torch.cuda.synchronize()
+    want = oracle_step(st, g, 1, 2, W.HYPERS)
+    for k in KEYS:
+        assert_same_bits(W.bits(arrays[k]), st[k], k)
+    got = e.read()
+    edq_close(got, want)
+    assert got["n"] == n
+    B.plan_destroy(plan)
+    del arrays, rows
+    torch.cuda.empty_cache()
+
+
+def test_gpt2_small_hundred_steps_collage_light_sampled():
+    # config 1: 148 tensors, 124,439,808 parameters, multi-tensor Collage-light, 100 steps with fresh gradients
+    dev = torch.device("cuda")
+    shapes = W.gpt2_small_shapes()
+    rng = np.random.default_rng(1)
+    tensors, rows, samples = [], [], []
+    for i, (_, n) in enumerate(shapes):
+        x = W.flat_weights(n, 1000 + i, dev)
+        d = dict(x_hi=x, x_lo=torch.zeros_like(x), m=torch.zeros_like(x), v_hi=torch.zeros_like(x),
+                 grad=torch.zeros_like(x))
+        tensors.append(d)
+        rows.append((d["x_hi"], d["x_lo"], d["m"], d["v_hi"], None, d["grad"], n))
+        wins = _windows(n, rng, 1024, 3)
+        st = {k: (_gather(d[k], wins) if k in d else None) for k in KEYS}
+        samples.append((wins, st))
+    plan = B.plan_create(rows)
+    e = EdqBuffers()
+    hyp = W.HYPERS
+    edq_hist = []
+    for t in range(1, 101):
+        for i, (_, n) in enumerate(shapes):
+            tensors[i]["grad"].copy_(W.normal_bf16(n, 1e-3, 2000 * 1000 + t * 1000 + i, dev))
+        B.adamw_step_multi(plan, e.hyper(hyp), t, B.LIGHT)
+        for i, (wins, st) in enumerate(samples):
+            oracle_step(st, _gather(tensors[i]["grad"], wins), t, 1, hyp, threads=1)
+        edq_hist.append(e.read()["edq"])
+        if t in (1, 2, 10, 50, 100):
+            for i, (wins, st) in enumerate(samples):
+                for k in ("x_hi", "x_lo", "m", "v_hi"):
+                    assert_same_bits(_gather(tensors[i][k], wins), st[k], f"step {t} {shapes[i][0]} {k}")
+    assert all(np.isfinite(edq_hist)) and min(edq_hist) > 0
+    assert B.pipeline_fault() == 0
+    B.plan_destroy(plan)
+
+
+def test_stress_set_collage_plus_against_plain_bf16():
+    # config 2: 64 Mi parameters, theta = +-U(0.5, 4), log-uniform gradients, lr 1e-5: whole arrays for the first
+    # steps, then a fixed 256 Ki slice for 300 steps; Collage-plus keeps what plain bfloat16 loses
+    dev = torch.device("cuda")
+    n, hyp = 1 << 26, W.HYPERS_STRESS
+    lo, hi = 12_345_672, 12_345_672 + (1 << 18)
+    theta = W.stress_weights(n, 2, dev)
+    state, host, edq = {}, {}, {}
+    for s in (2, 0):
+        z = lambda: torch.zeros_like(theta)
+        state[s] = dict(x_hi=theta.clone(), x_lo=z() if s else None, m=z(), v_hi=z(), v_lo=z() if s == 2 else None)
+        host[s] = {k: (W.bits(v) if v is not None else None) for k, v in state[s].items()}
+        edq[s] = []
+    e = EdqBuffers()
+    for t in range(1, 301):
+        g = W.stress_grads(n, 2, t, dev)
+        whole = t <= 2
+        gb = W.bits(g) if whole else W.bits(W.stress_grads(hi - lo, 2, t, "cpu", offset=lo))
+        if not whole and t == 3:          # from here on the oracle follows the slice only
+            host = {s: {k: (v[lo:hi].copy() if v is not None else None) for k, v in host[s].items()} for s in host}
+        if t in (3, 100, 300):
+            assert np.array_equal(gb, W.bits(g[lo:hi]))              # the slice generator reproduces the full one
+        for s in (2, 0):
+            d = state[s]
+            B.adamw_step(d["x_hi"], d["x_lo"], d["m"], d["v_hi"], d["v_lo"], g, n, e.hyper(hyp), t, s)
+            torch.cuda.synchronize()
+            edq[s].append(e.read())
+            want = oracle_step(host[s], gb, t, s, hyp)
+            if whole:
+                edq_close(edq[s][-1], want)
+            if whole or t in (3, 50, 150, 300):
+                for k in KEYS:
+                    if host[s][k] is not None:
+                        got = W.bits(d[k]) if whole else W.bits(d[k][lo:hi])
+                        assert_same_bits(got, host[s][k], f"strategy {s} step {t} {k}")
+    # most updates fall below half an ulp of theta: plain bfloat16 drops them from the first step on; the
+    # expansion carries them until its second component has grown to ~2^8 updates (a length-2 bfloat16
+    # expansion resolves ~2^-17 of theta), after which part of them is lost there too
+    assert edq[0][0]["lost"] > 0.5 * n and edq[0][-1]["lost"] > 0.5 * n
+    assert edq[2][19]["lost"] < 0.05 * n
+    assert edq[2][-1]["lost"] < edq[0][-1]["lost"]
+    assert all(c["edq"] >= a["edq"] for c, a in zip(edq[2], edq[0]))
+    assert B.pipeline_fault() == 0
+
+
+@pytest.mark.parametrize("strategy", [1, 2])
+def test_size_sweep_powers_of_four(strategy):
+    # config 4: flat tensors of 4^6 ... 4^12 parameters, two steps each, every array and EDQ
+    dev = torch.device("cuda")
+    hyp = W.HYPERS
+    for p in range(6, 13):
+        n = 4 ** p
+        theta = W.flat_weights(n, 4, dev)
+        z = lambda: torch.zeros_like(theta)
+        d = dict(x_hi=theta, x_lo=z(), m=z(), v_hi=z(), v_lo=z() if strategy == 2 else None)
+        st = {k: (W.bits(v) if v is not None else None) for k, v in d.items()}
+        e = EdqBuffers()
+        for t in (1, 2):
+            g = W.flat_grads(n, 4, t, dev)
+            B.adamw_step(d["x_hi"], d["x_lo"], d["m"], d["v_hi"], d["v_lo"], g, n, e.hyper(hyp), t, strategy)
+            torch.cuda.synchronize()
+            want = oracle_step(st, W.bits(g), t, strategy, hyp)
+            for k in KEYS:
+                if st[k] is not None:
+                    assert_same_bits(W.bits(d[k]), st[k], f"n=4^{p} step {t} {k}")
+            edq_close(e.read(), want)
