@@ -141,7 +141,7 @@ def run_collage(args):
 
     hyp = W.HYPERS
     arrays, rows, n = build_llama7b_state(torch, W, device, seed=3 + rank, layers=args.layers)
-    plan = B.plan_create(rows)
+    plan = B.plan_create(rows, args.chunk_elems)
     edq_dev = torch.zeros(64, dtype=torch.uint8, device=device)
     ws = torch.empty(B.workspace_bytes(), dtype=torch.uint8, device=device)
     edq_sums = edq_dev[:16].view(torch.float64)         # {dot, sumsq}: what ranks exchange
@@ -256,6 +256,51 @@ def run_e2e(torch, B, W, device, args):
                       "collage_adamw_step_host (768 MiB device staging)"}
 
 
+def run_size_sweep(args):
+    """Flat tensors of 4^6 ... 4^15 parameters (Collage-light and -plus, EDQ on): one JSON line per size.
+
+    Sizes whose state fits in L2 are rotated over enough independent buffer sets to exceed 512 MB, so
+    that "HBM GB/s" is not an L2 number; the smallest sizes are launch-latency bound and say so.
+    """
+    import torch
+    from paper_2405_03637_b200 import binding as B
+    from paper_2405_03637_b200 import workloads as W
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    peak, _ = measured_hbm_peak()
+    edq_dev = torch.zeros(64, dtype=torch.uint8, device=device)
+    ws = torch.empty(B.workspace_bytes(), dtype=torch.uint8, device=device)
+    stream = torch.cuda.current_stream()
+    for p in range(6, 16):
+        n = 4 ** p
+        for strategy, name in ((1, "collage_light"), (2, "collage_plus")):
+            state_bytes = (10 if strategy == 1 else 12) * n
+            sets = max(1, min(64, -(-(512 << 20) // state_bytes)))
+            bufs = []
+            for k in range(sets):
+                x = W.flat_weights(n, 4 + k, device)
+                z = lambda: torch.zeros_like(x)
+                bufs.append((x, z(), z(), z(), z() if strategy == 2 else None, W.flat_grads(n, 4 + k, 1, device)))
+            h = B.make_hyper(**W.HYPERS, edq_out=edq_dev, workspace=ws)
+            iters = max(20, min(400, int(2e10 // (n * BYTES_PER_PARAM[strategy])) * 4))
+            for t in range(1, 4):
+                B.adamw_step(*bufs[t % sets], n, h, t, strategy, stream)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for i in range(iters):
+                B.adamw_step(*bufs[i % sets], n, h, 4 + i, strategy, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / iters
+            gbs = n * BYTES_PER_PARAM[strategy] / (ms * 1e-3) / 1e9
+            print(json.dumps({"n": n, "strategy": name, "us_per_step": ms * 1e3, "params_per_sec": n / (ms * 1e-3),
+                              "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak, "frac_of_nominal_8TBps": gbs / 8000.0,
+                              "buffer_sets": sets, "launches_per_step": 2}), flush=True)
+            del bufs
+            torch.cuda.empty_cache()
+
+
 def run_cpu_baseline(W, seconds=15.0, threads=None):
     """The oracle as it stands on this machine's cores, on a bounded slice of the same workload."""
     import numpy as np
@@ -321,8 +366,12 @@ def main():
     ap.add_argument("--layers", type=int, default=32, help="transformer layers of the 7B-shaped set (32 = full)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--skip-extras", action="store_true", help="no e2e and no CPU baseline (profiling runs)")
+    ap.add_argument("--chunk-elems", type=int, default=0, help="chunk size of the multi-tensor plan (0 = library default)")
+    ap.add_argument("--size-sweep", action="store_true", help="flat-tensor size sweep instead of the benchmark")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.size_sweep:
+        run_size_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_collage(args)

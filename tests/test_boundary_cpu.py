@@ -117,7 +117,7 @@ def test_argument_errors_are_reported_before_any_cuda_call(L):
     assert L.collage_plan_create(t, 2, 0, ctypes.byref(plan)) == B.ERR_ALIAS
     assert L.collage_adamw_step_multi(None, ctypes.byref(ok), 1, 0, None) == B.ERR_NULL
     assert L.collage_plan_destroy(None) == B.OK
-    for s in range(7):
+    for s in range(8):
         assert B.status_string(s)
 
 

@@ -55,7 +55,7 @@ def test_ragged_tensor_set(strategy, chunk):
     host, dev, grads, rows = _build(shapes, strategy, seed=3, misalign_of=lambda i: (0, 0, 1, 0, 0, 3)[i % 6])
     plan = B.plan_create(rows, chunk)
     assert B.plan_num_elements(plan) == sum(n for _, n in shapes)
-    ce = chunk or 16384
+    ce = chunk or 24576
     assert B.plan_num_chunks(plan) == sum(-(-n // ce) for _, n in shapes)
     e = EdqBuffers()
     for t in (1, 2, 3):
