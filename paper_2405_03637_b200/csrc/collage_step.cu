@@ -399,27 +399,34 @@ static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t s
     auto kernel = adamw_step_pipeline_kernel<STRATEGY, EDQ, FLAT, FAST, CONSUMERS, VPT, STAGES>;
     constexpr size_t smem = sizeof(PipeSmem<CONSUMERS, VPT, STAGES, STRATEGY>) + 128;
     constexpr int threads = CONSUMERS + 32;
-    static int blocks_per_sm = 0;   // per instantiation
-    if (blocks_per_sm == 0) {
+    // per instantiation and per device: the shared-memory opt-in is a per-device function attribute
+    static int per_device[64] = {};
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    if (per_device[device] == 0) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
         int b = 0;
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, threads, smem);
         if (e != cudaSuccess) return e;
-        blocks_per_sm = b > 0 ? b : 1;
+        per_device[device] = b > 0 ? b : 1;
     }
+    const int blocks_per_sm = per_device[device];
 #else
     constexpr int UNROLL = COLLAGE_UNROLL;
     auto kernel = adamw_step_kernel<STRATEGY, EDQ, FLAT, FAST, UNROLL>;
     constexpr size_t smem = 0;
     constexpr int threads = kThreads;
-    static int blocks_per_sm = 0;   // per instantiation
-    if (blocks_per_sm == 0) {
+    static int per_device[64] = {};
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    if (per_device[device] == 0) {
         int b = 0;
         const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, threads, 0);
         if (e != cudaSuccess) return e;
-        blocks_per_sm = b > 0 ? b : 1;
+        per_device[device] = b > 0 ? b : 1;
     }
+    const int blocks_per_sm = per_device[device];
 #endif
     uint64_t grid = static_cast<uint64_t>(sm_count) * blocks_per_sm;
     if (grid > p.num_chunks) grid = p.num_chunks;
