@@ -2,28 +2,21 @@
 // streams every state array exactly once, plus the entry points that launch it.
 //
 // Work is cut into chunks of `chunk_elems` consecutive elements of one tensor.  Thread block b
-// takes chunks b, b + grid, b + 2*grid, ...  Two kernels walk the chunks the same way:
-//   * step_pipeline.cuh (default): tiles are moved between global and shared memory by the bulk
-//     asynchronous copy engine, the threads compute out of shared memory;
-//   * adamw_step_kernel below (-DCOLLAGE_PLAIN_KERNEL): each thread loads 16-byte vectors into
-//     registers, computes, stores.
-// In both, a thread owns 8 consecutive elements (one 16-byte vector per state array) at a time;
-// tensors whose pointers are not all 16-byte aligned, and the last (<8) elements of a tensor, go
-// through an element-wise path that feeds the same arithmetic.  EDQ sums: float within a vector,
-// double per thread, fixed-order tree per block, one partial per block, summed by a one-block
-// finalize kernel.
+// takes chunks b, b + grid, b + 2*grid, ...  The kernel (step_pipeline.cuh) moves tiles between
+// global and shared memory with the bulk asynchronous copy engine; its threads compute out of
+// shared memory, 8 consecutive elements (one 16-byte vector per state array) at a time.  Tensors
+// whose pointers are not all 16-byte aligned, and the ragged end of a tensor, go through plain or
+// element-wise accesses that feed the same arithmetic.  EDQ sums: float within a vector, double
+// per thread, fixed-order tree per block, one partial per block, summed by a one-block finalize
+// kernel.
 #include "host_common.cuh"
 #include "mcf_device.cuh"
 
-namespace collage {
-
-// Default data movement: the bulk-copy pipeline of step_pipeline.cuh.  Measured on B200 (2^30
-// parameters, Collage-plus with EDQ, median of 80 launches): 512 consumer threads + one producer warp,
-// one block per SM, three stages of 4096-element tiles reached 6.47 TB/s; the register-staged kernel
-// below (-DCOLLAGE_PLAIN_KERNEL) 6.07 TB/s; smaller tiles, more stages or two blocks per SM were slower.
-#ifndef COLLAGE_PLAIN_KERNEL
-#define COLLAGE_USE_PIPELINE 1
-#endif
+// Geometry of the pipeline kernel.  Measured on B200 (2^30 parameters, Collage-plus with EDQ, median
+// of 80 launches): 512 consumer threads + one producer warp, one block per SM, three stages of
+// 4096-element tiles reached 6.47 TB/s; an earlier register-staged kernel (16-byte loads into
+// registers, 6 blocks of 128 threads per SM) 6.07 TB/s; smaller tiles, more stages or two blocks
+// per SM were slower.
 #ifndef COLLAGE_PIPE_CONSUMERS
 #define COLLAGE_PIPE_CONSUMERS 512
 #endif
@@ -41,18 +34,9 @@ namespace collage {
 #ifndef COLLAGE_PIPE_MINBLOCKS
 #define COLLAGE_PIPE_MINBLOCKS 1
 #endif
-// Launch geometry of the register-staged kernel (128 threads x 6 resident blocks per SM, one
-// 8-element vector per thread in flight, 80 registers, was the fastest of the shapes tried).
-#ifndef COLLAGE_THREADS
-#define COLLAGE_THREADS 128
-#endif
-#ifndef COLLAGE_UNROLL
-#define COLLAGE_UNROLL 1
-#endif
-#ifndef COLLAGE_MINBLOCKS
-#define COLLAGE_MINBLOCKS 6
-#endif
-constexpr int kThreads = COLLAGE_THREADS;
+
+namespace collage {
+
 constexpr uint32_t kDefaultChunk = 24576;   // a whole number of tiles for every precision option (6 x 4096, 4 x 6144)
 // elements per tile of the pipeline kernel for a precision option
 constexpr uint32_t pipe_tile(int strategy) {
@@ -86,39 +70,9 @@ struct StepParams {
     EdqPartial* partials;       // one per block, or nullptr
 };
 
-// ---- 16-byte streaming accesses (each byte is touched once: do not keep it in L1) ----------
-#ifndef COLLAGE_LD_POLICY
-#define COLLAGE_LD_POLICY 0
-#endif
-#ifndef COLLAGE_ST_POLICY
-#define COLLAGE_ST_POLICY 0
-#endif
-__device__ __forceinline__ uint4 ld_stream(const uint16_t* p) {
-#if COLLAGE_LD_POLICY == 0
-    return __ldcs(reinterpret_cast<const uint4*>(p));
-#elif COLLAGE_LD_POLICY == 1
-    return *reinterpret_cast<const uint4*>(p);
-#elif COLLAGE_LD_POLICY == 2
-    uint4 v;
-    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-#else
-    uint4 v;
-    asm volatile("ld.global.L1::no_allocate.L2::evict_first.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
-#endif
-}
-__device__ __forceinline__ void st_stream(uint16_t* p, const uint4& v) {
-#if COLLAGE_ST_POLICY == 0
-    __stcs(reinterpret_cast<uint4*>(p), v);
-#elif COLLAGE_ST_POLICY == 1
-    *reinterpret_cast<uint4*>(p) = v;
-#elif COLLAGE_ST_POLICY == 2
-    __stwt(reinterpret_cast<uint4*>(p), v);
-#else
-    asm volatile("st.global.L1::no_allocate.L2::evict_first.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-#endif
-}
+// ---- 16-byte streaming accesses for tiles that bypass the copy pipeline ---------------------
+__device__ __forceinline__ uint4 ld_stream(const uint16_t* p) { return __ldcs(reinterpret_cast<const uint4*>(p)); }
+__device__ __forceinline__ void st_stream(uint16_t* p, const uint4& v) { __stcs(reinterpret_cast<uint4*>(p), v); }
 
 // element-wise gather/scatter of up to 8 bfloat16 values into / out of four packed registers
 __device__ __forceinline__ uint4 ld_elems(const uint16_t* p, int count) {
@@ -150,10 +104,6 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
     uint32_t* dv = reinterpret_cast<uint32_t*>(&s.dv);
     const uint32_t* g = reinterpret_cast<const uint32_t*>(&s.g);
     EdqAcc acc = {0ull, 0ull, 0u};
-#ifdef COLLAGE_NULL_COMPUTE
-    th[0] ^= g[0] & 1u;   // data-movement experiment only: no arithmetic
-    return;
-#endif
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         ElemState e;
@@ -226,88 +176,6 @@ __device__ __forceinline__ void store_elems(const Vec& s, const TensorRec& t, ui
 }  // namespace collage
 #include "step_pipeline.cuh"
 namespace collage {
-
-template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, int UNROLL>
-__global__ void __launch_bounds__(kThreads, COLLAGE_MINBLOCKS) adamw_step_kernel(const __grid_constant__ StepParams p) {
-    double dot = 0.0, sq = 0.0;
-    uint32_t lost = 0;
-    const StepScalars& k = p.k;
-
-    for (uint64_t c = blockIdx.x; c < p.num_chunks; c += gridDim.x) {
-        TensorRec t;
-        uint64_t start;
-        if (FLAT) {
-            t = p.flat;
-            start = c * p.chunk_elems;
-        } else {
-            const ChunkRec cr = p.chunks[c];
-            t = p.tensors[cr.tensor];
-            start = static_cast<uint64_t>(cr.index) * p.chunk_elems;
-        }
-        const uint64_t left = t.n - start;
-        const uint32_t len = left < p.chunk_elems ? static_cast<uint32_t>(left) : p.chunk_elems;
-        const uint32_t nvec = len >> 3;
-        const int rem = static_cast<int>(len & 7u);
-
-        if (t.aligned) {
-            for (uint32_t i = threadIdx.x; i < nvec; i += kThreads * UNROLL) {
-                Vec s[UNROLL];
-#pragma unroll
-                for (int u = 0; u < UNROLL; ++u)
-                    if (i + u * kThreads < nvec) load_vec<STRATEGY>(s[u], t, start + 8ull * (i + u * kThreads));
-#pragma unroll
-                for (int u = 0; u < UNROLL; ++u)
-                    if (i + u * kThreads < nvec) {
-                        compute_vec<STRATEGY, EDQ, FAST>(s[u], k, 8, dot, sq, lost);
-                        store_vec<STRATEGY>(s[u], t, start + 8ull * (i + u * kThreads));
-                    }
-            }
-        } else {
-            for (uint32_t i = threadIdx.x; i < nvec; i += kThreads) {
-                Vec s;
-                load_elems<STRATEGY>(s, t, start + 8ull * i, 8);
-                compute_vec<STRATEGY, EDQ, FAST>(s, k, 8, dot, sq, lost);
-                store_elems<STRATEGY>(s, t, start + 8ull * i, 8);
-            }
-        }
-        if (rem && threadIdx.x == (nvec % kThreads)) {
-            Vec s;
-            load_elems<STRATEGY>(s, t, start + 8ull * nvec, rem);
-            compute_vec<STRATEGY, EDQ, FAST>(s, k, rem, dot, sq, lost);
-            store_elems<STRATEGY>(s, t, start + 8ull * nvec, rem);
-        }
-    }
-
-    if (EDQ) {
-        unsigned long long lost64 = lost;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            dot += __shfl_down_sync(0xFFFFFFFFu, dot, o);
-            sq += __shfl_down_sync(0xFFFFFFFFu, sq, o);
-            lost64 += __shfl_down_sync(0xFFFFFFFFu, lost64, o);
-        }
-        __shared__ double s_dot[kThreads / 32], s_sq[kThreads / 32];
-        __shared__ unsigned long long s_lost[kThreads / 32];
-        const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-        if (lane == 0) {
-            s_dot[warp] = dot;
-            s_sq[warp] = sq;
-            s_lost[warp] = lost64;
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            double d = 0.0, q = 0.0;
-            unsigned long long l = 0;
-#pragma unroll
-            for (int w = 0; w < kThreads / 32; ++w) {
-                d += s_dot[w];
-                q += s_sq[w];
-                l += s_lost[w];
-            }
-            p.partials[blockIdx.x] = EdqPartial{d, q, l, 0ull};
-        }
-    }
-}
 
 // Sums the per-block partials in a fixed order and writes the EDQ record (Eq. 3).
 // With `accumulate` the sums are added to the record's current contents (a step issued in slabs).
@@ -393,7 +261,6 @@ static collage_status_t make_scalars(const collage_hyper_t* hyper, uint64_t step
 
 template <int STRATEGY, bool EDQ, bool FLAT, bool FAST>
 static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t stream, int* grid_out) {
-#ifdef COLLAGE_USE_PIPELINE
     constexpr int CONSUMERS = STRATEGY == 0 ? COLLAGE_PIPE_CONSUMERS_A : COLLAGE_PIPE_CONSUMERS;
     constexpr int VPT = COLLAGE_PIPE_VPT, STAGES = COLLAGE_PIPE_STAGES;
     auto kernel = adamw_step_pipeline_kernel<STRATEGY, EDQ, FLAT, FAST, CONSUMERS, VPT, STAGES>;
@@ -411,24 +278,7 @@ static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t s
         if (e != cudaSuccess) return e;
         per_device[device] = b > 0 ? b : 1;
     }
-    const int blocks_per_sm = per_device[device];
-#else
-    constexpr int UNROLL = COLLAGE_UNROLL;
-    auto kernel = adamw_step_kernel<STRATEGY, EDQ, FLAT, FAST, UNROLL>;
-    constexpr size_t smem = 0;
-    constexpr int threads = kThreads;
-    static int per_device[64] = {};
-    int device = 0;
-    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return cudaErrorInvalidDevice;
-    if (per_device[device] == 0) {
-        int b = 0;
-        const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, threads, 0);
-        if (e != cudaSuccess) return e;
-        per_device[device] = b > 0 ? b : 1;
-    }
-    const int blocks_per_sm = per_device[device];
-#endif
-    uint64_t grid = static_cast<uint64_t>(sm_count) * blocks_per_sm;
+    uint64_t grid = static_cast<uint64_t>(sm_count) * per_device[device];
     if (grid > p.num_chunks) grid = p.num_chunks;
     if (grid > static_cast<uint64_t>(kMaxGrid)) grid = kMaxGrid;
     *grid_out = static_cast<int>(grid);
@@ -476,11 +326,7 @@ static cudaError_t launch_flat(void* x_hi, void* x_lo, void* m, void* v_hi, void
                      aligned16(grad);
     // four tiles per chunk when there is plenty of work, one tile per chunk when the tensor is small,
     // so that every SM still gets a share
-#ifdef COLLAGE_USE_PIPELINE
     const uint32_t tile = pipe_tile(strategy);
-#else
-    const uint32_t tile = kDefaultChunk / 4;
-#endif
     uint32_t chunk = 4 * tile;
     if ((n + chunk - 1) / chunk < 4ull * static_cast<uint64_t>(sm_count)) chunk = tile;
     p.chunk_elems = chunk;

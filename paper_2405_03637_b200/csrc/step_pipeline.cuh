@@ -1,7 +1,7 @@
-// Bulk-copy pipelined variant of the fused AdamW step.
+// The fused AdamW step kernel: a bulk-copy pipeline around the arithmetic of mcf_device.cuh.
 //
-// Same arithmetic and same chunk walk as adamw_step_kernel, different data movement: one
-// producer thread per block moves whole tiles (kTile elements of every state array) between
+// Each block walks its chunks of the chunk table (or of the one flat tensor).  One producer
+// thread per block moves whole tiles (kTile elements of every state array) between
 // global and shared memory with the bulk asynchronous copy engine (cp.async.bulk, completion on
 // an mbarrier), kStages tiles deep, while the consumer warps compute out of shared memory and
 // write their results back into the same shared slots, from where the producer bulk-stores them.
