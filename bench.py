@@ -148,8 +148,15 @@ def run_collage(args):
     edq_lost = edq_dev[32:40].view(torch.int64)         # lost-update count
     stream = torch.cuda.current_stream()
 
+    if args.per_tensor:                                 # variant: EDQ kept per tensor (three launches per step)
+        per = torch.zeros(len(rows) * 40, dtype=torch.uint8, device=device)
+        cws = torch.empty(B.plan_workspace_bytes(plan), dtype=torch.uint8, device=device)
+
     def step(t):
-        B.adamw_step_multi(plan, B.make_hyper(**hyp, edq_out=edq_dev, workspace=ws), t, STRATEGY, stream)
+        if args.per_tensor:
+            B.adamw_step_multi_per_tensor(plan, B.make_hyper(**hyp, edq_out=edq_dev), t, STRATEGY, per, len(rows), cws, stream)
+        else:
+            B.adamw_step_multi(plan, B.make_hyper(**hyp, edq_out=edq_dev, workspace=ws), t, STRATEGY, stream)
         if world > 1:                                   # EDQ is global: sum the partial sums over ranks
             dist.all_reduce(edq_sums)
             dist.all_reduce(edq_lost)
@@ -196,7 +203,7 @@ def run_collage(args):
                    "state_bytes_per_param": 12, "hbm_bytes_per_param_per_step": BYTES_PER_PARAM[STRATEGY],
                    "edq": True, "l2": "state (80.9 GB per GPU) far exceeds the 126 MB L2; no flush needed",
                    "parallelism": f"dp{world} (each rank owns a full 7B-shaped shard; EDQ sums all-reduced)"},
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": (3 if args.per_tensor else 2) * args.steps,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_BYTES_PER_PARAM * n / 1e9, "traffic_unit": "GB per launch (ncu, scaled by parameters)",
                      "algorithmic": n * BYTES_PER_PARAM[STRATEGY] / 1e9, "peak_source": peak_src, "frac_of_nominal_8TBps": achieved / 8000.0,
@@ -367,6 +374,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--skip-extras", action="store_true", help="no e2e and no CPU baseline (profiling runs)")
     ap.add_argument("--chunk-elems", type=int, default=0, help="chunk size of the multi-tensor plan (0 = library default)")
+    ap.add_argument("--per-tensor", action="store_true", help="time the per-tensor EDQ variant of the step")
     ap.add_argument("--size-sweep", action="store_true", help="flat-tensor size sweep instead of the benchmark")
     args = ap.parse_args()
     if args.size_sweep:

@@ -150,6 +150,26 @@ collage_status_t collage_plan_create(const collage_tensor_t* tensors, int num, u
 collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const collage_hyper_t* hyper,
                                           uint64_t step, collage_strategy_t strategy, void* stream);
 collage_status_t collage_plan_destroy(collage_plan_t* plan);
+
+/* The multi-tensor step with EDQ kept per tensor (Eq. 2-3 evaluated on each parameter tensor of the
+ * plan separately; the lost-update count of Def. 3.2 per tensor gives the imprecision percentage of
+ * Figure 3, left).  Same state update as collage_adamw_step_multi, bit for bit.
+ *   per_tensor_out_dev : DEVICE collage_edq_t[num], num = the `num` given to collage_plan_create;
+ *                        entry i belongs to tensors[i] (all zero for an empty tensor).
+ *   chunk_workspace    : DEVICE scratch of at least collage_plan_workspace_bytes(plan) bytes, 16-byte
+ *                        aligned (32 bytes per chunk of the plan).
+ *   hyper->edq_out     : optional DEVICE collage_edq_t for the whole plan = the per-tensor sums added
+ *                        in tensor order (association differs from collage_adamw_step_multi's, so
+ *                        the last bits may differ); hyper->workspace is not used by this call.
+ * Three launches (step, per-tensor sums, total) instead of two.
+ * Errors: as collage_adamw_step_multi, plus ERR_ARG when num differs from the plan's and
+ * ERR_WORKSPACE for the chunk workspace. */
+size_t collage_plan_workspace_bytes(const collage_plan_t* plan);
+collage_status_t collage_adamw_step_multi_per_tensor(const collage_plan_t* plan, const collage_hyper_t* hyper,
+                                                     uint64_t step, collage_strategy_t strategy,
+                                                     collage_edq_t* per_tensor_out_dev, int num,
+                                                     void* chunk_workspace, size_t chunk_workspace_bytes,
+                                                     void* stream);
 /* Plan facts for callers that report or shard: total elements, number of chunks. */
 uint64_t collage_plan_num_elements(const collage_plan_t* plan);
 uint64_t collage_plan_num_chunks(const collage_plan_t* plan);

@@ -21,7 +21,8 @@ EXPORTS = (
     "collage_status_string", "collage_derive_scalars", "collage_workspace_bytes", "collage_adamw_step",
     "collage_adamw_step_host",
     "collage_plan_create", "collage_adamw_step_multi", "collage_plan_destroy", "collage_plan_num_elements",
-    "collage_plan_num_chunks", "collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_grow",
+    "collage_plan_num_chunks", "collage_plan_workspace_bytes", "collage_adamw_step_multi_per_tensor",
+    "collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_grow",
     "collage_scaling", "collage_mul", "collage_renormalize", "collage_rounded_op", "collage_edq",
     "collage_selftest", "collage_pipeline_fault", "collage_edq_static",
 )
@@ -80,6 +81,10 @@ def lib() -> ctypes.CDLL:
         L.collage_plan_num_elements.argtypes = [vp]
         L.collage_plan_num_chunks.restype = u64
         L.collage_plan_num_chunks.argtypes = [vp]
+        L.collage_plan_workspace_bytes.restype = ctypes.c_size_t
+        L.collage_plan_workspace_bytes.argtypes = [vp]
+        L.collage_adamw_step_multi_per_tensor.argtypes = [vp, ctypes.POINTER(Hyper), u64, i32, vp, i32, vp,
+                                                          ctypes.c_size_t, vp]
         for name in ("collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_renormalize"):
             getattr(L, name).argtypes = [vp, vp, vp, vp, u64, vp]
         L.collage_grow.argtypes = [vp, vp, vp, vp, vp, u64, vp]
@@ -154,6 +159,29 @@ def plan_create(tensors, chunk_elems: int = 0) -> int:
 def adamw_step_multi(plan: int, hyper: Hyper, step: int, strategy: int, stream=None):
     _check(lib().collage_adamw_step_multi(plan, ctypes.byref(hyper), step, strategy, _ptr(stream)),
            "collage_adamw_step_multi")
+
+
+def plan_workspace_bytes(plan: int) -> int:
+    return int(lib().collage_plan_workspace_bytes(plan))
+
+
+def adamw_step_multi_per_tensor(plan: int, hyper: Hyper, step: int, strategy: int, per_tensor_out, num: int,
+                                chunk_workspace, stream=None):
+    """per_tensor_out: CUDA uint8 tensor of num * 40 bytes; chunk_workspace: CUDA uint8 tensor."""
+    _check(lib().collage_adamw_step_multi_per_tensor(plan, ctypes.byref(hyper), step, strategy, _ptr(per_tensor_out), num,
+                                                     _ptr(chunk_workspace),
+                                                     chunk_workspace.numel() * chunk_workspace.element_size(),
+                                                     _ptr(stream)), "collage_adamw_step_multi_per_tensor")
+
+
+def read_edq_array(dev_bytes, num: int) -> list:
+    """Decode num consecutive device collage_edq_t records."""
+    raw = dev_bytes.detach().cpu().numpy().tobytes()
+    out = []
+    for i in range(num):
+        rec = Edq.from_buffer_copy(raw[i * ctypes.sizeof(Edq):(i + 1) * ctypes.sizeof(Edq)])
+        out.append(dict(dot=rec.dot, sumsq=rec.sumsq, edq=rec.edq, n=int(rec.n), lost=int(rec.lost)))
+    return out
 
 
 def plan_destroy(plan: int):

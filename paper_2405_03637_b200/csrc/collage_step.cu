@@ -68,6 +68,7 @@ struct StepParams {
     uint32_t chunk_elems;
     StepScalars k;
     EdqPartial* partials;       // one per block, or nullptr
+    EdqPartial* chunk_partials; // one per chunk (per-tensor EDQ), or nullptr
 };
 
 // ---- 16-byte streaming accesses for tiles that bypass the copy pipeline ---------------------
@@ -219,6 +220,61 @@ __global__ void __launch_bounds__(256) edq_finalize_kernel(const EdqPartial* par
     }
 }
 
+// Per-tensor EDQ: block t adds the per-chunk partials of tensor t (chunks first[t] .. first[t+1]-1)
+// in a fixed order and writes record index[t]; a second, single-block kernel adds the records.
+__global__ void __launch_bounds__(256) edq_per_tensor_kernel(const EdqPartial* chunk_partials, const uint64_t* first,
+                                                             const uint32_t* index, const uint64_t* sizes,
+                                                             collage_edq_t* out) {
+    __shared__ double s_dot[256], s_sq[256];
+    __shared__ unsigned long long s_lost[256];
+    const uint64_t lo = first[blockIdx.x], hi = first[blockIdx.x + 1];
+    double d = 0.0, q = 0.0;
+    unsigned long long l = 0;
+    for (uint64_t i = lo + threadIdx.x; i < hi; i += 256) {
+        d += chunk_partials[i].dot;
+        q += chunk_partials[i].sq;
+        l += chunk_partials[i].lost;
+    }
+    s_dot[threadIdx.x] = d;
+    s_sq[threadIdx.x] = q;
+    s_lost[threadIdx.x] = l;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) {
+            s_dot[threadIdx.x] += s_dot[threadIdx.x + o];
+            s_sq[threadIdx.x] += s_sq[threadIdx.x + o];
+            s_lost[threadIdx.x] += s_lost[threadIdx.x + o];
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        collage_edq_t r;
+        r.dot = s_dot[0];
+        r.sumsq = s_sq[0];
+        r.edq = s_sq[0] > 0.0 ? s_dot[0] / sqrt(s_sq[0]) : 0.0;
+        r.n = sizes[blockIdx.x];
+        r.lost = s_lost[0];
+        out[index[blockIdx.x]] = r;
+    }
+}
+
+__global__ void __launch_bounds__(32) edq_sum_records_kernel(const collage_edq_t* records, int count, collage_edq_t* out) {
+    if (threadIdx.x != 0) return;
+    double d = 0.0, q = 0.0;
+    unsigned long long l = 0, n = 0;
+    for (int i = 0; i < count; ++i) {      // tensor order: deterministic
+        d += records[i].dot;
+        q += records[i].sumsq;
+        l += records[i].lost;
+        n += records[i].n;
+    }
+    out->dot = d;
+    out->sumsq = q;
+    out->edq = q > 0.0 ? d / sqrt(q) : 0.0;
+    out->n = n;
+    out->lost = l;
+}
+
 void launch_edq_finalize(const EdqPartial* partials, int count, uint64_t n, collage_edq_t* out, cudaStream_t stream,
                          bool accumulate) {
     edq_finalize_kernel<<<1, 256, 0, stream>>>(partials, count, n, out, accumulate ? 1 : 0);
@@ -259,11 +315,11 @@ static collage_status_t make_scalars(const collage_hyper_t* hyper, uint64_t step
     return COLLAGE_OK;
 }
 
-template <int STRATEGY, bool EDQ, bool FLAT, bool FAST>
+template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, bool PER_CHUNK = false>
 static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t stream, int* grid_out) {
     constexpr int CONSUMERS = STRATEGY == 0 ? COLLAGE_PIPE_CONSUMERS_A : COLLAGE_PIPE_CONSUMERS;
     constexpr int VPT = COLLAGE_PIPE_VPT, STAGES = COLLAGE_PIPE_STAGES;
-    auto kernel = adamw_step_pipeline_kernel<STRATEGY, EDQ, FLAT, FAST, CONSUMERS, VPT, STAGES>;
+    auto kernel = adamw_step_pipeline_kernel<STRATEGY, EDQ, FLAT, FAST, CONSUMERS, VPT, STAGES, PER_CHUNK>;
     constexpr size_t smem = sizeof(PipeSmem<CONSUMERS, VPT, STAGES, STRATEGY>) + 128;
     constexpr int threads = CONSUMERS + 32;
     // per instantiation and per device: the shared-memory opt-in is a per-device function attribute
@@ -298,6 +354,19 @@ static cudaError_t dispatch_step2(const StepParams& p, int strategy, bool edq, i
         default: return launch_step<2, true, FLAT, FAST>(p, sm_count, stream, grid_out);
     }
 }
+// multi-tensor step with one EDQ record per chunk
+static cudaError_t dispatch_step_per_chunk(const StepParams& p, int strategy, int sm_count, cudaStream_t stream,
+                                           int* grid_out) {
+    switch (strategy * 2 + (p.k.fast ? 1 : 0)) {
+        case 0: return launch_step<0, true, false, false, true>(p, sm_count, stream, grid_out);
+        case 1: return launch_step<0, true, false, true, true>(p, sm_count, stream, grid_out);
+        case 2: return launch_step<1, true, false, false, true>(p, sm_count, stream, grid_out);
+        case 3: return launch_step<1, true, false, true, true>(p, sm_count, stream, grid_out);
+        case 4: return launch_step<2, true, false, false, true>(p, sm_count, stream, grid_out);
+        default: return launch_step<2, true, false, true, true>(p, sm_count, stream, grid_out);
+    }
+}
+
 template <bool FLAT>
 static cudaError_t dispatch_step(const StepParams& p, int strategy, bool edq, int sm_count, cudaStream_t stream,
                                  int* grid_out) {
@@ -355,6 +424,10 @@ using namespace collage;
 struct collage_plan {
     TensorRec* d_tensors = nullptr;
     ChunkRec* d_chunks = nullptr;
+    uint64_t* d_first_chunk = nullptr;   // per non-empty tensor, plus an end marker
+    uint64_t* d_sizes = nullptr;         // per non-empty tensor
+    uint32_t* d_orig_index = nullptr;    // position of the tensor in the caller's array
+    int num_given = 0;                   // length of the caller's array
     uint64_t num_chunks = 0;
     uint64_t num_elements = 0;
     uint32_t chunk_elems = 0;
@@ -446,6 +519,8 @@ collage_status_t collage_plan_create(const collage_tensor_t* tensors, int num, u
     std::vector<TensorRec> recs;
     std::vector<ChunkRec> chunks;
     std::vector<ByteRange> ranges;
+    std::vector<uint64_t> first_chunk, sizes;
+    std::vector<uint32_t> orig_index;
     bool has_x_lo = true, has_v_lo = true;
     uint64_t total = 0;
     for (int i = 0; i < num; ++i) {
@@ -472,13 +547,18 @@ collage_status_t collage_plan_create(const collage_tensor_t* tensors, int num, u
         const uint64_t nchunks = (t.n + chunk_elems - 1) / chunk_elems;
         if (nchunks > 0xFFFFFFFFull || chunks.size() + nchunks > 0xFFFFFFFFull) return COLLAGE_ERR_ARG;
         const uint32_t id = static_cast<uint32_t>(recs.size());
+        first_chunk.push_back(chunks.size());
+        sizes.push_back(t.n);
+        orig_index.push_back(static_cast<uint32_t>(i));
         for (uint64_t c = 0; c < nchunks; ++c) chunks.push_back({id, static_cast<uint32_t>(c)});
         recs.push_back(r);
         total += t.n;
     }
     if (any_overlap(ranges)) return COLLAGE_ERR_ALIAS;
+    first_chunk.push_back(chunks.size());
 
     collage_plan* plan = new collage_plan;
+    plan->num_given = num;
     plan->num_chunks = chunks.size();
     plan->num_elements = total;
     plan->chunk_elems = chunk_elems;
@@ -492,9 +572,21 @@ collage_status_t collage_plan_create(const collage_tensor_t* tensors, int num, u
             cudaMemcpy(plan->d_tensors, recs.data(), recs.size() * sizeof(TensorRec), cudaMemcpyHostToDevice) !=
                 cudaSuccess ||
             cudaMemcpy(plan->d_chunks, chunks.data(), chunks.size() * sizeof(ChunkRec), cudaMemcpyHostToDevice) !=
-                cudaSuccess) {
+                cudaSuccess ||
+            cudaMalloc(&plan->d_first_chunk, first_chunk.size() * sizeof(uint64_t)) != cudaSuccess ||
+            cudaMalloc(&plan->d_sizes, sizes.size() * sizeof(uint64_t)) != cudaSuccess ||
+            cudaMalloc(&plan->d_orig_index, orig_index.size() * sizeof(uint32_t)) != cudaSuccess ||
+            cudaMemcpy(plan->d_first_chunk, first_chunk.data(), first_chunk.size() * sizeof(uint64_t),
+                       cudaMemcpyHostToDevice) != cudaSuccess ||
+            cudaMemcpy(plan->d_sizes, sizes.data(), sizes.size() * sizeof(uint64_t), cudaMemcpyHostToDevice) !=
+                cudaSuccess ||
+            cudaMemcpy(plan->d_orig_index, orig_index.data(), orig_index.size() * sizeof(uint32_t),
+                       cudaMemcpyHostToDevice) != cudaSuccess) {
             cudaFree(plan->d_tensors);
             cudaFree(plan->d_chunks);
+            cudaFree(plan->d_first_chunk);
+            cudaFree(plan->d_sizes);
+            cudaFree(plan->d_orig_index);
             delete plan;
             return COLLAGE_ERR_CUDA;
         }
@@ -535,11 +627,65 @@ collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const coll
     return COLLAGE_OK;
 }
 
+size_t collage_plan_workspace_bytes(const collage_plan_t* plan) {
+    return plan ? static_cast<size_t>(plan->num_chunks) * sizeof(EdqPartial) + sizeof(EdqPartial) : 0;
+}
+
+collage_status_t collage_adamw_step_multi_per_tensor(const collage_plan_t* plan, const collage_hyper_t* hyper,
+                                                     uint64_t step, collage_strategy_t strategy,
+                                                     collage_edq_t* per_tensor_out_dev, int num,
+                                                     void* chunk_workspace, size_t chunk_workspace_bytes,
+                                                     void* stream) {
+    if (!plan || !hyper || !per_tensor_out_dev) return COLLAGE_ERR_NULL;
+    collage_hyper_t h = *hyper;
+    void* global_out = h.edq_out;
+    h.edq_out = nullptr;                      // the block-partial workspace of the plain multi step is not used
+    collage_status_t st = check_common(&h, step, strategy);
+    if (st != COLLAGE_OK) return st;
+    if (num != plan->num_given) return COLLAGE_ERR_ARG;
+    if (strategy >= COLLAGE_LIGHT && !plan->has_x_lo) return COLLAGE_ERR_NULL;
+    if (strategy == COLLAGE_PLUS && !plan->has_v_lo) return COLLAGE_ERR_NULL;
+    if (!chunk_workspace || (reinterpret_cast<uintptr_t>(chunk_workspace) & 15u) ||
+        chunk_workspace_bytes < collage_plan_workspace_bytes(plan))
+        return COLLAGE_ERR_WORKSPACE;
+    DeviceInfo dev;
+    st = current_device(&dev);
+    if (st != COLLAGE_OK) return st;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+
+    StepParams p{};
+    st = make_scalars(&h, step, &p.k);
+    if (st != COLLAGE_OK) return st;
+    p.tensors = plan->d_tensors;
+    p.chunks = plan->d_chunks;
+    p.num_chunks = plan->num_chunks;
+    p.chunk_elems = plan->chunk_elems;
+    p.chunk_partials = static_cast<EdqPartial*>(chunk_workspace);
+    if (num > 0 && cudaMemsetAsync(per_tensor_out_dev, 0, static_cast<size_t>(num) * sizeof(collage_edq_t), cs) != cudaSuccess)
+        return COLLAGE_ERR_CUDA;
+    if (plan->num_chunks > 0) {
+        int grid = 0;
+        if (dispatch_step_per_chunk(p, strategy, dev.sm_count, cs, &grid) != cudaSuccess) return COLLAGE_ERR_CUDA;
+        edq_per_tensor_kernel<<<plan->num_tensors, 256, 0, cs>>>(p.chunk_partials, plan->d_first_chunk, plan->d_orig_index,
+                                                                 plan->d_sizes, per_tensor_out_dev);
+        if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
+    }
+    if (global_out) {
+        edq_sum_records_kernel<<<1, 32, 0, cs>>>(per_tensor_out_dev, num, static_cast<collage_edq_t*>(global_out));
+        if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
+    }
+    return COLLAGE_OK;
+}
+
 collage_status_t collage_plan_destroy(collage_plan_t* plan) {
     if (!plan) return COLLAGE_OK;
-    cudaError_t a = cudaFree(plan->d_tensors), b = cudaFree(plan->d_chunks);
+    bool ok = cudaFree(plan->d_tensors) == cudaSuccess;
+    ok = (cudaFree(plan->d_chunks) == cudaSuccess) && ok;
+    ok = (cudaFree(plan->d_first_chunk) == cudaSuccess) && ok;
+    ok = (cudaFree(plan->d_sizes) == cudaSuccess) && ok;
+    ok = (cudaFree(plan->d_orig_index) == cudaSuccess) && ok;
     delete plan;
-    return (a == cudaSuccess && b == cudaSuccess) ? COLLAGE_OK : COLLAGE_ERR_CUDA;
+    return ok ? COLLAGE_OK : COLLAGE_ERR_CUDA;
 }
 
 uint64_t collage_plan_num_elements(const collage_plan_t* plan) { return plan ? plan->num_elements : 0; }

@@ -101,11 +101,14 @@ struct PipeSmem {
     alignas(128) uint16_t data[STAGES][ArrayCount<STRATEGY>::kIn][kTile];
     alignas(8) uint64_t full[STAGES];
     alignas(8) uint64_t done[STAGES];
+    alignas(8) uint64_t red_full, red_free;   // hand-over of per-chunk EDQ sums (PER_CHUNK only)
     double red_dot[CONSUMERS / 32], red_sq[CONSUMERS / 32];
     unsigned long long red_lost[CONSUMERS / 32];
 };
 
-template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, int CONSUMERS, int VPT, int STAGES>
+// PER_CHUNK: the EDQ sums are written once per chunk (p.chunk_partials[chunk]) instead of once per
+// block, so that a later kernel can add them up tensor by tensor.
+template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, int CONSUMERS, int VPT, int STAGES, bool PER_CHUNK = false>
 __global__ void __launch_bounds__(CONSUMERS + 32, COLLAGE_PIPE_MINBLOCKS)
 adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
     constexpr int kTile = CONSUMERS * 8 * VPT;
@@ -122,6 +125,8 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
             pipe::mbar_init(&sm.full[s], 1);
             pipe::mbar_init(&sm.done[s], kWarps);
         }
+        pipe::mbar_init(&sm.red_full, kWarps);
+        pipe::mbar_init(&sm.red_free, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
@@ -205,6 +210,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
         }
     } else {
         const int lane = threadIdx.x & 31;
+        uint32_t chunks_done = 0;
         for (uint64_t c = blockIdx.x; c < p.num_chunks && alive; c += gridDim.x) {
             TensorRec t;
             uint64_t start;
@@ -220,7 +226,8 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
             const uint32_t len = left < p.chunk_elems ? static_cast<uint32_t>(left) : p.chunk_elems;
             for (uint32_t off = 0; off < len; off += kTile, ++it) {
                 const int s = it % STAGES;
-                alive = pipe::mbar_wait(&sm.full[s], (it / STAGES) & 1u, 40u + s);
+                // a wait that gives up must take the whole warp with it (the lanes meet again in __syncwarp)
+                alive = __all_sync(0xFFFFFFFFu, pipe::mbar_wait(&sm.full[s], (it / STAGES) & 1u, 40u + s));
                 if (!alive) break;
                 const uint32_t tl = (len - off) < static_cast<uint32_t>(kTile) ? (len - off) : kTile;
                 if (t.aligned && tl == static_cast<uint32_t>(kTile)) {
@@ -267,10 +274,51 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                 __syncwarp();
                 if (lane == 0) pipe::mbar_arrive(&sm.done[s]);
             }
+            if (EDQ && PER_CHUNK && alive) {
+                // One record per chunk, summed over the consumers in a fixed order.  The hand-over of the
+                // per-warp sums goes through two mbarriers with bounded waits (never a bar.sync, which
+                // could not time out): red_full = "all warps have written", red_free = "thread 0 has read".
+                unsigned long long lost64 = lost;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    dot += __shfl_down_sync(0xFFFFFFFFu, dot, o);
+                    sq += __shfl_down_sync(0xFFFFFFFFu, sq, o);
+                    lost64 += __shfl_down_sync(0xFFFFFFFFu, lost64, o);
+                }
+                if (chunks_done > 0)
+                    alive = __all_sync(0xFFFFFFFFu, pipe::mbar_wait(&sm.red_free, (chunks_done - 1) & 1u, 50u));
+                if (alive) {
+                    if (lane == 0) {
+                        sm.red_dot[threadIdx.x >> 5] = dot;
+                        sm.red_sq[threadIdx.x >> 5] = sq;
+                        sm.red_lost[threadIdx.x >> 5] = lost64;
+                        pipe::mbar_arrive(&sm.red_full);
+                    }
+                    if (threadIdx.x == 0) {
+                        if (pipe::mbar_wait(&sm.red_full, chunks_done & 1u, 51u)) {
+                            double d = 0.0, q = 0.0;
+                            unsigned long long l = 0;
+#pragma unroll
+                            for (int w = 0; w < kWarps; ++w) {
+                                d += sm.red_dot[w];
+                                q += sm.red_sq[w];
+                                l += sm.red_lost[w];
+                            }
+                            p.chunk_partials[c] = EdqPartial{d, q, l, 0ull};
+                            pipe::mbar_arrive(&sm.red_free);
+                        }
+                    }
+                    __syncwarp();
+                }
+                dot = 0.0;
+                sq = 0.0;
+                lost = 0;
+                ++chunks_done;
+            }
         }
     }
 
-    if (EDQ) {
+    if (EDQ && !PER_CHUNK) {
         unsigned long long lost64 = lost;
         if (!is_producer) {
 #pragma unroll

@@ -113,3 +113,49 @@ def test_plan_strategy_needs_its_components():
     torch.cuda.synchronize()
     assert e.read()["edq"] == 0.0 and e.read()["n"] == 0
     B.plan_destroy(empty)
+
+
+@pytest.mark.parametrize("strategy", [0, 1, 2])
+@pytest.mark.parametrize("chunk", [0, 2048])
+def test_per_tensor_edq_matches_oracle_tensor_by_tensor(strategy, chunk):
+    shapes = W.ragged_shapes() + [("big", 700_001)]
+    hyp = W.HYPERS
+    host, dev, grads, rows = _build(shapes, strategy, seed=7, misalign_of=lambda i: (0, 1, 0)[i % 3])
+    plan = B.plan_create(rows, chunk)
+    num = len(shapes)
+    per = torch.zeros(num * 40, dtype=torch.uint8, device="cuda")
+    cws = torch.empty(B.plan_workspace_bytes(plan), dtype=torch.uint8, device="cuda")
+    assert B.plan_workspace_bytes(plan) >= 32 * B.plan_num_chunks(plan)
+    total = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    for t in (1, 2, 3):
+        gbits = _set_grads(shapes, grads, 7, t)
+        h = B.make_hyper(**hyp, edq_out=total)
+        B.adamw_step_multi_per_tensor(plan, h, t, strategy, per, num, cws)
+        torch.cuda.synchronize()
+        recs = B.read_edq_array(per, num)
+        tot = dict(dot=0.0, sumsq=0.0, lost=0)
+        for i, (st, g) in enumerate(zip(host, gbits)):
+            if g.size == 0:
+                assert recs[i] == dict(dot=0.0, sumsq=0.0, edq=0.0, n=0, lost=0)
+                continue
+            want = oracle_step(st, g, t, strategy, hyp, threads=1)
+            edq_close(recs[i], want)
+            assert recs[i]["n"] == g.size
+            for k in KEYS:
+                if st[k] is not None:
+                    assert_same_bits(dev[i][k].bits(), st[k], f"tensor {i} {k} step {t}")
+                    assert dev[i][k].guards_intact()
+            tot["dot"] += want["dot"]; tot["sumsq"] += want["sumsq"]; tot["lost"] += want["lost"]
+        tot["edq"] = tot["dot"] / np.sqrt(tot["sumsq"])
+        got = B.read_edq(total)
+        edq_close(got, tot)
+        assert got["n"] == sum(n for _, n in shapes)
+    assert B.pipeline_fault() == 0
+    # argument checks
+    with pytest.raises(B.CollageError) as err:
+        B.adamw_step_multi_per_tensor(plan, B.make_hyper(**hyp), 1, strategy, per, num - 1, cws)
+    assert err.value.status == B.ERR_ARG
+    with pytest.raises(B.CollageError) as err:
+        B.adamw_step_multi_per_tensor(plan, B.make_hyper(**hyp), 1, strategy, per, num, cws[:64])
+    assert err.value.status == B.ERR_WORKSPACE
+    B.plan_destroy(plan)
