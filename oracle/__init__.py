@@ -22,7 +22,10 @@ _LIB = _HERE / "liboracle_collage.so"
 STRATEGY_BF16 = 0   # option A
 STRATEGY_LIGHT = 1  # option B
 STRATEGY_PLUS = 2   # option C
+STRATEGY_KAHAN = 3  # BF16-Kahan comparator (Appendix B): x_lo holds the compensation c
 FLAG_EPS_INSIDE_SQRT = 1
+FLAG_TWOSUM_GROW = 2     # parameter Grow built on TwoSum (Appendix C)
+FLAG_DECAY_BY_GROW = 4   # weight decay applied by an addition of its own (Appendix D)
 
 OP_ADD, OP_SUB, OP_MUL, OP_DIV, OP_SQRT, OP_FMA = range(6)
 

@@ -201,8 +201,15 @@ scalars derive_scalars(double lr, double beta1, double beta2, double eps, double
     return s;
 }
 
-enum { STRAT_BF16 = 0, STRAT_LIGHT = 1, STRAT_PLUS = 2 };
-enum { FLAG_EPS_INSIDE_SQRT = 1 };
+enum { STRAT_BF16 = 0, STRAT_LIGHT = 1, STRAT_PLUS = 2, STRAT_KAHAN = 3 };
+enum { FLAG_EPS_INSIDE_SQRT = 1, FLAG_TWOSUM_GROW = 2, FLAG_DECAY_BY_GROW = 4 };
+
+// Grow with TwoSum in place of Fast2Sum (Appendix C: TwoSum yields the same expansion for any
+// a, b without sorting): exact also where |x| < |a|.
+inline pair16 grow_two_sum(pair16 xy, bf16 a) {
+    pair16 uv = two_sum(xy.hi, a);
+    return two_sum(uv.hi, op_add(xy.lo, uv.lo));
+}
 
 struct edq_sums { double dot, sumsq; uint64_t lost; };
 
@@ -235,26 +242,43 @@ inline void step_one(bf16& th, bf16* dth, bf16& m, bf16& v, bf16* dv, bf16 g,
     else den = op_add(op_sqrt(vhat), s.eps);
     const bf16 r = op_div(mhat, den);
     const bf16 w = op_mul(s.lam, th);          // decay uses the first component of theta (reading)
-    const bf16 u = op_add(r, w);
-    const bf16 delta = op_mul(op_neg(s.a), u);
+    // Appendix D, weight decay: either summed into the update (default, "the latter option"), or
+    // applied to the parameter by an addition of its own (flag): d = -a (*) (lam (*) theta).
+    const bool split_decay = (flags & FLAG_DECAY_BY_GROW) != 0;
+    const bf16 decay = op_mul(op_neg(s.a), w);
+    const bf16 delta = split_decay ? op_mul(op_neg(s.a), r) : op_mul(op_neg(s.a), op_add(r, w));
     // line 13
     const bf16 th_old = th;
     const bf16 dth_old = dth ? *dth : 0;
-    if (strategy == STRAT_BF16) {
-        th = op_add(th, delta);                // Eq. 1
+    auto add_to_parameter = [&](bf16 upd) {
+        if (strategy == STRAT_BF16) {
+            th = op_add(th, upd);              // Eq. 1
+        } else {
+            pair16 nt = (flags & FLAG_TWOSUM_GROW) ? grow_two_sum(pair16{th, *dth}, upd) : grow(pair16{th, *dth}, upd);
+            th = nt.hi;
+            *dth = nt.lo;
+        }
+    };
+    if (strategy == STRAT_KAHAN) {
+        // Appendix B, Kahan summation: the compensation c (stored where dtheta would be) is added to the
+        // update, and c <- F(update (-) F(theta_t (-) theta_{t-1})) is kept for the next step
+        const bf16 comp = op_add(delta, *dth);
+        th = op_add(th_old, comp);
+        *dth = op_sub(comp, op_sub(th, th_old));
     } else {
-        pair16 nt = grow(pair16{th, *dth}, delta);
-        th = nt.hi;
-        *dth = nt.lo;
+        if (split_decay) add_to_parameter(decay);
+        add_to_parameter(delta);
     }
-    // Eq. 2 generalised to an expansion: effective update = (theta'+dtheta') - (theta+dtheta)
-    const double eff = (widen(th) - widen(th_old)) + (dth ? (widen(*dth) - widen(dth_old)) : 0.0);
-    const double d = widen(delta);
+    // Eq. 2 generalised to an expansion: effective update = (theta'+dtheta') - (theta+dtheta).  For Kahan
+    // the parameter is theta alone (Eq. 2 as printed); c is bookkeeping, not part of the value.
+    const bool pair_value = dth && strategy != STRAT_KAHAN;
+    const double eff = (widen(th) - widen(th_old)) + (pair_value ? (widen(*dth) - widen(dth_old)) : 0.0);
+    const double d = widen(delta) + (split_decay ? widen(decay) : 0.0);      // intended update
     acc.dot += d * eff;
     acc.sumsq += d * d;
     // lost arithmetic (Def. 3.2; "not updated", Figure 3 left): an update was intended and the stored
     // parameter (every component, compared as values) is what it was
-    const bool unchanged = widen(th) == widen(th_old) && (!dth || widen(*dth) == widen(dth_old));
+    const bool unchanged = widen(th) == widen(th_old) && (!pair_value || widen(*dth) == widen(dth_old));
     if (d != 0.0 && unchanged) acc.lost += 1;
     if (delta_out) *delta_out = delta;
 }

@@ -120,6 +120,49 @@ def scaling(v, a1, a2):
     return fast_two_sum(x, e)
 
 
+def two_sum(a, b):
+    x = add(a, b)
+    bv = sub(x, a)
+    av = sub(x, bv)
+    return x, add(sub(a, av), sub(b, bv))
+
+
+def grow_two_sum(x, y, a):
+    u, v = two_sum(x, a)
+    return two_sum(u, add(y, v))
+
+
+def adamw_element_variant(th, dth, m, v, dv, g, sc, strategy, twosum_grow=False, split_decay=False):
+    """Step variants: strategy 3 = BF16-Kahan (dth holds c); TwoSum-based Grow; decay by its own addition."""
+    m = add(mul(sc["b1"], m), mul(sc["c1"], g))
+    tv = mul(sc["c2"], mul(g, g))
+    if strategy == 2:
+        p, e = mcf_mul(sc["b2h"], sc["b2l"], v, dv)
+        v, dv = grow(p, e, tv)
+    else:
+        v = add(mul(sc["b2"], v), tv)
+    r = div(div(m, sc["bc1"]), add(sqrt(div(v, sc["bc2"])), sc["eps"]))
+    w = mul(sc["lam"], th)
+    nega = sc["a"] ^ 0x8000
+    decay = mul(nega, w)
+    delta = mul(nega, r) if split_decay else mul(nega, add(r, w))
+
+    def apply(th, dth, upd):
+        if strategy == 0:
+            return add(th, upd), dth
+        return grow_two_sum(th, dth, upd) if twosum_grow else grow(th, dth, upd)
+
+    if strategy == 3:
+        comp = add(delta, dth)
+        new = add(th, comp)
+        th, dth = new, sub(comp, sub(new, th))
+    else:
+        if split_decay:
+            th, dth = apply(th, dth, decay)
+        th, dth = apply(th, dth, delta)
+    return th, dth, m, v, dv, delta
+
+
 def adamw_element(th, dth, m, v, dv, g, sc, strategy, eps_inside=False):
     """Algorithm 2 lines 8-13 for one parameter; sc = dict of bfloat16 scalars. Returns new state and the update."""
     m = add(mul(sc["b1"], m), mul(sc["c1"], g))
