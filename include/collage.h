@@ -39,7 +39,7 @@ extern "C" {
 typedef enum {
     COLLAGE_OK = 0,
     COLLAGE_ERR_NULL = 1,       /* a required pointer is NULL                                   */
-    COLLAGE_ERR_ARG = 2,        /* step == 0, unknown strategy/op, hyper-parameter out of range */
+    COLLAGE_ERR_ARG = 2,        /* step == 0, unknown strategy/op/flag combination, hyper out of range */
     COLLAGE_ERR_ALIAS = 3,      /* two tensors of one call overlap                              */
     COLLAGE_ERR_ARCH = 4,       /* current device is not sm_100                                 */
     COLLAGE_ERR_CUDA = 5,       /* a CUDA runtime call or launch failed                         */
@@ -51,11 +51,24 @@ typedef enum {
 typedef enum {
     COLLAGE_BF16 = 0,   /* A: theta, m, v single bfloat16                    ( 8 B/param with grad) */
     COLLAGE_LIGHT = 1,  /* B: (theta, dtheta) pair                           (10 B/param)           */
-    COLLAGE_PLUS = 2    /* C: (theta, dtheta), (v, dv) pairs, beta2 as pair  (12 B/param)           */
+    COLLAGE_PLUS = 2,   /* C: (theta, dtheta), (v, dv) pairs, beta2 as pair  (12 B/param)           */
+    /* Comparator of the paper's experiments, not one of its options: BF16 AdamW with Kahan summation
+     * at the parameter update (Appendix B): update' = update (+) c; theta' = theta (+) update';
+     * c' = update' (-) (theta' (-) theta).  Same arrays as option B, x_lo holding c (10 B/param).
+     * EDQ counts theta alone (Eq. 2 as printed). */
+    COLLAGE_KAHAN = 3
 } collage_strategy_t;
 
 /* Algorithm 2 line 12 prints epsilon under the root; AdamW has it outside.  Default: outside. */
 #define COLLAGE_FLAG_EPS_INSIDE_SQRT 1u
+/* Variants of the parameter update (default: off).
+ * TWOSUM_GROW: line 13's Grow uses TwoSum instead of Fast2Sum (Appendix C: same expansion with no
+ *   ordering requirement), so the update is error-free also where |theta| < |update|.  B and C only.
+ * DECAY_BY_GROW: the weight decay is not summed into the update (Appendix D: "either ... or") but
+ *   applied first by an addition (Grow for B and C) of its own: d = (-a) (*) (lam (*) theta), then the
+ *   Adam part (-a) (*) r.  A, B, C.  EDQ then measures against d + update. */
+#define COLLAGE_FLAG_TWOSUM_GROW 2u
+#define COLLAGE_FLAG_DECAY_BY_GROW 4u
 
 /* Hyper-parameters of one step (Algorithm 2 line 1).  HOST struct.
  * Valid ranges: lr, eps, weight_decay >= 0 and finite; 0 <= beta1, beta2 < 1. */
@@ -109,7 +122,8 @@ collage_status_t collage_derive_scalars(const collage_hyper_t* hyper, uint64_t s
 size_t collage_workspace_bytes(uint64_t n_total);
 
 /* One AdamW step over one flat tensor (Algorithm 2 lines 8-13, all n parameters, step t >= 1).
- *   x_hi, m, v_hi, grad : required.   x_lo : required iff strategy != COLLAGE_BF16, else must
+ *   x_hi, m, v_hi, grad : required.   x_lo : required iff strategy != COLLAGE_BF16 (delta-theta, or
+ *   the Kahan compensation for COLLAGE_KAHAN), else must
  *   be NULL.   v_lo : required iff strategy == COLLAGE_PLUS, else must be NULL.
  * Errors: ERR_NULL, ERR_ARG (step 0, bad strategy, hyper range), ERR_ALIAS (overlapping
  * tensors), ERR_WORKSPACE (edq_out set, workspace too small), ERR_ARCH, ERR_CUDA. */
@@ -161,7 +175,8 @@ collage_status_t collage_plan_destroy(collage_plan_t* plan);
  *   hyper->edq_out     : optional DEVICE collage_edq_t for the whole plan = the per-tensor sums added
  *                        in tensor order (association differs from collage_adamw_step_multi's, so
  *                        the last bits may differ); hyper->workspace is not used by this call.
- * Three launches (step, per-tensor sums, total) instead of two.
+ * Three launches (step, per-tensor sums, total) instead of two.  The variant flags (TWOSUM_GROW,
+ * DECAY_BY_GROW) are not available through this entry point (ERR_ARG).
  * Errors: as collage_adamw_step_multi, plus ERR_ARG when num differs from the plan's and
  * ERR_WORKSPACE for the chunk workspace. */
 size_t collage_plan_workspace_bytes(const collage_plan_t* plan);

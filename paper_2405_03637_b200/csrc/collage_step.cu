@@ -95,7 +95,7 @@ struct Vec {
 };
 
 // The arithmetic of 8 parameters held in registers.  `valid` < 8 masks padded lanes out of EDQ.
-template <int STRATEGY, bool EDQ, bool FAST>
+template <int STRATEGY, bool EDQ, bool FAST, bool VARIANT = false>
 __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int valid, double& dot, double& sq,
                                             uint32_t& lost) {
     uint32_t* th = reinterpret_cast<uint32_t*>(&s.th);
@@ -109,27 +109,32 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
     for (int j = 0; j < 4; ++j) {
         ElemState e;
         e.th = th[j];
-        e.dth = STRATEGY >= 1 ? dth[j] : 0u;
+        e.dth = STRATEGY >= 1 ? dth[j] : 0u;   // delta-theta (B, C) or the Kahan compensation
         e.m = m[j];
         e.v = v[j];
         e.dv = STRATEGY == 2 ? dv[j] : 0u;
         const bf2 th_old = e.th, dth_old = e.dth;
-        bf2 delta = adamw_pair<STRATEGY, FAST>(e, g[j], k);
+        const PairUpdate up = adamw_pair<STRATEGY, FAST, VARIANT>(e, g[j], k);
         th[j] = e.th;
         m[j] = e.m;
         v[j] = e.v;
         if (STRATEGY >= 1) dth[j] = e.dth;
         if (STRATEGY == 2) dv[j] = e.dv;
         if (EDQ) {
-            bf2 th_new = e.th, dth_new = e.dth;
+            bf2 th_new = e.th, dth_new = e.dth, delta = up.delta, decay = up.decay;
             if (valid < 8) {            // padded lanes hold zeros on input; keep them out of the sums
                 const int lanes = valid - 2 * j;
                 const uint32_t mask = lanes >= 2 ? 0xFFFFFFFFu : (lanes == 1 ? 0x0000FFFFu : 0u);
                 delta &= mask;
+                decay &= mask;
                 th_new &= mask;
                 dth_new &= mask;
             }
-            edq_pair<(STRATEGY >= 1)>(acc, th_old, dth_old, th_new, dth_new, delta);
+            // intended update: line 12, plus the separate decay term when there is one
+            f32x2 d = widen2(delta);
+            if (VARIANT && (k.flags & 4u)) d = add_f32x2(d, widen2(decay));
+            // the stored parameter is the pair for options B and C, theta alone for A and Kahan
+            edq_pair_f<(STRATEGY == 1 || STRATEGY == 2)>(acc, th_old, dth_old, th_new, dth_new, d);
         }
     }
     if (EDQ) {
@@ -315,11 +320,11 @@ static collage_status_t make_scalars(const collage_hyper_t* hyper, uint64_t step
     return COLLAGE_OK;
 }
 
-template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, bool PER_CHUNK = false>
+template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, bool PER_CHUNK = false, bool VARIANT = false>
 static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t stream, int* grid_out) {
     constexpr int CONSUMERS = STRATEGY == 0 ? COLLAGE_PIPE_CONSUMERS_A : COLLAGE_PIPE_CONSUMERS;
     constexpr int VPT = COLLAGE_PIPE_VPT, STAGES = COLLAGE_PIPE_STAGES;
-    auto kernel = adamw_step_pipeline_kernel<STRATEGY, EDQ, FLAT, FAST, CONSUMERS, VPT, STAGES, PER_CHUNK>;
+    auto kernel = adamw_step_pipeline_kernel<STRATEGY, EDQ, FLAT, FAST, CONSUMERS, VPT, STAGES, PER_CHUNK, VARIANT>;
     constexpr size_t smem = sizeof(PipeSmem<CONSUMERS, VPT, STAGES, STRATEGY>) + 128;
     constexpr int threads = CONSUMERS + 32;
     // per instantiation and per device: the shared-memory opt-in is a per-device function attribute
@@ -351,7 +356,9 @@ static cudaError_t dispatch_step2(const StepParams& p, int strategy, bool edq, i
         case 2: return launch_step<1, false, FLAT, FAST>(p, sm_count, stream, grid_out);
         case 3: return launch_step<1, true, FLAT, FAST>(p, sm_count, stream, grid_out);
         case 4: return launch_step<2, false, FLAT, FAST>(p, sm_count, stream, grid_out);
-        default: return launch_step<2, true, FLAT, FAST>(p, sm_count, stream, grid_out);
+        case 5: return launch_step<2, true, FLAT, FAST>(p, sm_count, stream, grid_out);
+        case 6: return launch_step<3, false, FLAT, FAST>(p, sm_count, stream, grid_out);
+        default: return launch_step<3, true, FLAT, FAST>(p, sm_count, stream, grid_out);
     }
 }
 // multi-tensor step with one EDQ record per chunk
@@ -363,13 +370,33 @@ static cudaError_t dispatch_step_per_chunk(const StepParams& p, int strategy, in
         case 2: return launch_step<1, true, false, false, true>(p, sm_count, stream, grid_out);
         case 3: return launch_step<1, true, false, true, true>(p, sm_count, stream, grid_out);
         case 4: return launch_step<2, true, false, false, true>(p, sm_count, stream, grid_out);
-        default: return launch_step<2, true, false, true, true>(p, sm_count, stream, grid_out);
+        case 5: return launch_step<2, true, false, true, true>(p, sm_count, stream, grid_out);
+        case 6: return launch_step<3, true, false, false, true>(p, sm_count, stream, grid_out);
+        default: return launch_step<3, true, false, true, true>(p, sm_count, stream, grid_out);
+    }
+}
+
+// steps with a variant flag set (TwoSum Grow, decay by its own addition): options A, B, C
+template <bool FLAT, bool FAST>
+static cudaError_t dispatch_variant(const StepParams& p, int strategy, bool edq, int sm_count, cudaStream_t stream,
+                                    int* grid_out) {
+    switch (strategy * 2 + (edq ? 1 : 0)) {
+        case 0: return launch_step<0, false, FLAT, FAST, false, true>(p, sm_count, stream, grid_out);
+        case 1: return launch_step<0, true, FLAT, FAST, false, true>(p, sm_count, stream, grid_out);
+        case 2: return launch_step<1, false, FLAT, FAST, false, true>(p, sm_count, stream, grid_out);
+        case 3: return launch_step<1, true, FLAT, FAST, false, true>(p, sm_count, stream, grid_out);
+        case 4: return launch_step<2, false, FLAT, FAST, false, true>(p, sm_count, stream, grid_out);
+        case 5: return launch_step<2, true, FLAT, FAST, false, true>(p, sm_count, stream, grid_out);
+        default: return cudaErrorInvalidValue;
     }
 }
 
 template <bool FLAT>
 static cudaError_t dispatch_step(const StepParams& p, int strategy, bool edq, int sm_count, cudaStream_t stream,
                                  int* grid_out) {
+    if (p.k.flags & (COLLAGE_FLAG_TWOSUM_GROW | COLLAGE_FLAG_DECAY_BY_GROW))
+        return p.k.fast ? dispatch_variant<FLAT, true>(p, strategy, edq, sm_count, stream, grid_out)
+                        : dispatch_variant<FLAT, false>(p, strategy, edq, sm_count, stream, grid_out);
     return p.k.fast ? dispatch_step2<FLAT, true>(p, strategy, edq, sm_count, stream, grid_out)
                     : dispatch_step2<FLAT, false>(p, strategy, edq, sm_count, stream, grid_out);
 }
@@ -407,9 +434,14 @@ static cudaError_t launch_flat(void* x_hi, void* x_lo, void* m, void* v_hi, void
 static collage_status_t check_common(const collage_hyper_t* hyper, uint64_t step, int strategy) {
     if (!hyper) return COLLAGE_ERR_NULL;
     if (step == 0) return COLLAGE_ERR_ARG;
-    if (strategy < COLLAGE_BF16 || strategy > COLLAGE_PLUS) return COLLAGE_ERR_ARG;
+    if (strategy < COLLAGE_BF16 || strategy > COLLAGE_KAHAN) return COLLAGE_ERR_ARG;
     if (!hyper_in_range(hyper)) return COLLAGE_ERR_ARG;
-    if (hyper->flags & ~COLLAGE_FLAG_EPS_INSIDE_SQRT) return COLLAGE_ERR_ARG;
+    if (hyper->flags & ~(COLLAGE_FLAG_EPS_INSIDE_SQRT | COLLAGE_FLAG_TWOSUM_GROW | COLLAGE_FLAG_DECAY_BY_GROW))
+        return COLLAGE_ERR_ARG;
+    // TwoSum Grow needs a parameter pair (B, C); the Kahan comparator takes neither variant
+    if ((hyper->flags & COLLAGE_FLAG_TWOSUM_GROW) && strategy != COLLAGE_LIGHT && strategy != COLLAGE_PLUS)
+        return COLLAGE_ERR_ARG;
+    if ((hyper->flags & COLLAGE_FLAG_DECAY_BY_GROW) && strategy == COLLAGE_KAHAN) return COLLAGE_ERR_ARG;
     if (hyper->edq_out) {
         if (!hyper->workspace || hyper->workspace_bytes < kWorkspaceBytes) return COLLAGE_ERR_WORKSPACE;
         if (reinterpret_cast<uintptr_t>(hyper->workspace) & 15u) return COLLAGE_ERR_WORKSPACE;
@@ -643,6 +675,7 @@ collage_status_t collage_adamw_step_multi_per_tensor(const collage_plan_t* plan,
     collage_status_t st = check_common(&h, step, strategy);
     if (st != COLLAGE_OK) return st;
     if (num != plan->num_given) return COLLAGE_ERR_ARG;
+    if (h.flags & (COLLAGE_FLAG_TWOSUM_GROW | COLLAGE_FLAG_DECAY_BY_GROW)) return COLLAGE_ERR_ARG;   // not built
     if (strategy >= COLLAGE_LIGHT && !plan->has_x_lo) return COLLAGE_ERR_NULL;
     if (strategy == COLLAGE_PLUS && !plan->has_v_lo) return COLLAGE_ERR_NULL;
     if (!chunk_workspace || (reinterpret_cast<uintptr_t>(chunk_workspace) & 15u) ||

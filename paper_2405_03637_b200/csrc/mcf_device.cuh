@@ -264,6 +264,12 @@ __device__ __forceinline__ bf2pair grow2(bf2 x, bf2 y, bf2 a) {
     return fast_two_sum2(s.hi, add2(y, s.lo));
 }
 
+// Grow with TwoSum in place of Fast2Sum (Appendix C): error-free for any ordering of |x| and |a|
+__device__ __forceinline__ bf2pair grow_two_sum2(bf2 x, bf2 y, bf2 a) {
+    const bf2pair s = two_sum2(x, a);
+    return two_sum2(s.hi, add2(y, s.lo));
+}
+
 // Algorithm Scaling: float v times expansion (a1, a2)
 __device__ __forceinline__ bf2pair scaling2(bf2 v, bf2 a1, bf2 a2) {
     const bf2pair p = two_prod2(a1, v);
@@ -291,7 +297,7 @@ struct StepScalars {
     bf2 neg_a;         // -RN(lr)
     bf2 lam;           // RN(weight_decay)
     bf2 eps;           // RN(eps)
-    uint32_t flags;    // bit 0: epsilon under the root
+    uint32_t flags;    // bit 0: epsilon under the root; bit 1: TwoSum Grow; bit 2: decay by its own addition
     uint32_t fast;     // host-checked: 2^-100 <= bc1, bc2 <= 1 and 2^-54 <= eps <= 2^60
 };
 
@@ -307,29 +313,34 @@ struct ElemState {
 // epsilon outside the root a subnormal v-hat may be flushed by the root approximation: its root is
 // below 2^-63 < ulp(eps)/2 and is absorbed by the addition of eps either way.
 template <bool FAST>
-__device__ __forceinline__ bf2 update_direction(bf2 m, bf2 v, bf2 th, const StepScalars& k) {
-    bf2 mhat, vhat, den, r;
+__device__ __forceinline__ bf2 update_ratio(bf2 m, bf2 v, const StepScalars& k) {
+    bf2 mhat, vhat, den;
     if (FAST) {
         mhat = div2_by_scalar(m, k.rbc1);
         vhat = div2_by_scalar(v, k.rbc2);
         if (k.flags & 1u) den = sqrt2_flushing(add2(vhat, k.eps));   // v-hat + eps >= eps: never subnormal
         else den = add2(sqrt2_flushing(vhat), k.eps);
-        r = div2_normal_divisor(mhat, den);
-    } else {
-        mhat = div2_scalar(m, k.bc1, k.rbc1);
-        vhat = div2_scalar(v, k.bc2, k.rbc2);
-        if (k.flags & 1u) den = sqrt2(add2(vhat, k.eps));
-        else den = add2(sqrt2(vhat), k.eps);
-        r = div2(mhat, den);
+        return div2_normal_divisor(mhat, den);
     }
-    const bf2 u = add2(r, mul2(k.lam, th));
-    return mul2(k.neg_a, u);
+    mhat = div2_scalar(m, k.bc1, k.rbc1);
+    vhat = div2_scalar(v, k.bc2, k.rbc2);
+    if (k.flags & 1u) den = sqrt2(add2(vhat, k.eps));
+    else den = add2(sqrt2(vhat), k.eps);
+    return div2(mhat, den);
 }
 
-// Algorithm 2 lines 8-13 for two parameters.  STRATEGY: 0 = A, 1 = B, 2 = C.  Returns the
-// bfloat16 update of line 12; `s` is updated in place.
-template <int STRATEGY, bool FAST>
-__device__ __forceinline__ bf2 adamw_pair(ElemState& s, bf2 g, const StepScalars& k) {
+// What one step asked of two parameters: the update of line 12 and, when weight decay is applied
+// by an addition of its own (Appendix D; flags bit 2), that decay term.
+struct PairUpdate {
+    bf2 delta, decay;
+};
+
+// Algorithm 2 lines 8-13 for two parameters; `s` is updated in place.
+// STRATEGY: 0 = A, 1 = B, 2 = C, 3 = BF16-Kahan (Appendix B; s.dth holds the compensation c).
+// VARIANT kernels honour flags bit 1 (the parameter Grow uses TwoSum) and bit 2 (decay by its own
+// addition); the others are compiled without either, so the common path carries no test for them.
+template <int STRATEGY, bool FAST, bool VARIANT>
+__device__ __forceinline__ PairUpdate adamw_pair(ElemState& s, bf2 g, const StepScalars& k) {
     // line 8
     s.m = add2(mul2(k.b1, s.m), mul2(k.c1, g));
     // line 9
@@ -343,16 +354,33 @@ __device__ __forceinline__ bf2 adamw_pair(ElemState& s, bf2 g, const StepScalars
         s.v = add2(mul2(k.b2, s.v), tv);
     }
     // lines 10-12
-    const bf2 delta = update_direction<FAST>(s.m, s.v, s.th, k);
+    const bf2 r = update_ratio<FAST>(s.m, s.v, k);
+    const bf2 w = mul2(k.lam, s.th);
+    const bool split_decay = VARIANT && (k.flags & 4u) != 0;
+    PairUpdate up;
+    up.decay = split_decay ? mul2(k.neg_a, w) : 0u;
+    up.delta = split_decay ? mul2(k.neg_a, r) : mul2(k.neg_a, add2(r, w));
     // line 13
-    if (STRATEGY == 0) {
-        s.th = add2(s.th, delta);
+    if (STRATEGY == 3) {
+        const bf2 comp = add2(up.delta, s.dth);
+        const bf2 th_new = add2(s.th, comp);
+        s.dth = sub2(comp, sub2(th_new, s.th));
+        s.th = th_new;
+    } else if (STRATEGY == 0) {
+        if (split_decay) s.th = add2(s.th, up.decay);
+        s.th = add2(s.th, up.delta);
     } else {
-        const bf2pair nt = grow2(s.th, s.dth, delta);
+        const bool two_sum = VARIANT && (k.flags & 2u) != 0;
+        if (split_decay) {
+            const bf2pair nd = two_sum ? grow_two_sum2(s.th, s.dth, up.decay) : grow2(s.th, s.dth, up.decay);
+            s.th = nd.hi;
+            s.dth = nd.lo;
+        }
+        const bf2pair nt = two_sum ? grow_two_sum2(s.th, s.dth, up.delta) : grow2(s.th, s.dth, up.delta);
         s.th = nt.hi;
         s.dth = nt.lo;
     }
-    return delta;
+    return up;
 }
 
 // EDQ contributions of two parameters (Eq. 2-3): differences, products and running sums in
@@ -362,9 +390,10 @@ struct EdqAcc {
     uint32_t lost;
 };
 
+// `d` is the intended update as two floats; the stored parameter is (th, dth) when HAS_LO, else th alone.
 template <bool HAS_LO>
-__device__ __forceinline__ void edq_pair(EdqAcc& acc, bf2 th_old, bf2 dth_old, bf2 th_new, bf2 dth_new, bf2 delta) {
-    const f32x2 d = widen2(delta), o = widen2(th_old), n = widen2(th_new);
+__device__ __forceinline__ void edq_pair_f(EdqAcc& acc, bf2 th_old, bf2 dth_old, bf2 th_new, bf2 dth_new, f32x2 d) {
+    const f32x2 o = widen2(th_old), n = widen2(th_new);
     f32x2 e = sub_f32x2(n, o);
     bool same0 = lo_of(n) == lo_of(o), same1 = hi_of(n) == hi_of(o);
     if (HAS_LO) {
@@ -377,6 +406,10 @@ __device__ __forceinline__ void edq_pair(EdqAcc& acc, bf2 th_old, bf2 dth_old, b
     acc.sq = fma_f32x2(d, d, acc.sq);
     acc.lost += (lo_of(d) != 0.0f && same0) ? 1u : 0u;
     acc.lost += (hi_of(d) != 0.0f && same1) ? 1u : 0u;
+}
+template <bool HAS_LO>
+__device__ __forceinline__ void edq_pair(EdqAcc& acc, bf2 th_old, bf2 dth_old, bf2 th_new, bf2 dth_new, bf2 delta) {
+    edq_pair_f<HAS_LO>(acc, th_old, dth_old, th_new, dth_new, widen2(delta));
 }
 __device__ __forceinline__ float edq_dot(const EdqAcc& a) { return __fadd_rn(lo_of(a.dot), hi_of(a.dot)); }
 __device__ __forceinline__ float edq_sq(const EdqAcc& a) { return __fadd_rn(lo_of(a.sq), hi_of(a.sq)); }

@@ -108,7 +108,8 @@ struct PipeSmem {
 
 // PER_CHUNK: the EDQ sums are written once per chunk (p.chunk_partials[chunk]) instead of once per
 // block, so that a later kernel can add them up tensor by tensor.
-template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, int CONSUMERS, int VPT, int STAGES, bool PER_CHUNK = false>
+template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, int CONSUMERS, int VPT, int STAGES, bool PER_CHUNK = false,
+          bool VARIANT = false>
 __global__ void __launch_bounds__(CONSUMERS + 32, COLLAGE_PIPE_MINBLOCKS)
 adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
     constexpr int kTile = CONSUMERS * 8 * VPT;
@@ -242,7 +243,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                         if (STRATEGY >= 1) v.dth = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
                         if (STRATEGY == 2) v.dv = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
                         v.g = *reinterpret_cast<const uint4*>(&sm.data[s][a][e]);
-                        compute_vec<STRATEGY, EDQ, FAST>(v, k, 8, dot, sq, lost);
+                        compute_vec<STRATEGY, EDQ, FAST, VARIANT>(v, k, 8, dot, sq, lost);
                         a = 0;
                         *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.th;
                         *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.m;
@@ -260,14 +261,14 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                         Vec v;
                         if (t.aligned) load_vec<STRATEGY>(v, t, base + 8ull * i);
                         else load_elems<STRATEGY>(v, t, base + 8ull * i, 8);
-                        compute_vec<STRATEGY, EDQ, FAST>(v, k, 8, dot, sq, lost);
+                        compute_vec<STRATEGY, EDQ, FAST, VARIANT>(v, k, 8, dot, sq, lost);
                         if (t.aligned) store_vec<STRATEGY>(v, t, base + 8ull * i);
                         else store_elems<STRATEGY>(v, t, base + 8ull * i, 8);
                     }
                     if (rem && threadIdx.x == (nvec % CONSUMERS)) {
                         Vec v;
                         load_elems<STRATEGY>(v, t, base + 8ull * nvec, rem);
-                        compute_vec<STRATEGY, EDQ, FAST>(v, k, rem, dot, sq, lost);
+                        compute_vec<STRATEGY, EDQ, FAST, VARIANT>(v, k, rem, dot, sq, lost);
                         store_elems<STRATEGY>(v, t, base + 8ull * nvec, rem);
                     }
                 }

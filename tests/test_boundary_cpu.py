@@ -75,13 +75,18 @@ def test_argument_errors_are_reported_before_any_cuda_call(L):
                                              kw.get("strategy", B.BF16), None)
     assert L.collage_adamw_step(dummy, None, dummy, dummy, None, dummy, 16, None, 1, 0, None) == B.ERR_NULL
     assert call(step=0) == B.ERR_ARG
-    assert call(strategy=3) == B.ERR_ARG
+    assert call(strategy=4) == B.ERR_ARG
+    assert call(strategy=B.KAHAN) == B.ERR_NULL                      # the compensation array is missing
     assert call(strategy=-1) == B.ERR_ARG
     for bad in (dict(lr=-1.0), dict(beta1=1.0), dict(beta2=1.5), dict(eps=float("nan")), dict(weight_decay=float("inf"))):
         kw = dict(lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
         kw.update(bad)
         assert call(hyper=B.make_hyper(**kw)) == B.ERR_ARG
     assert call(hyper=B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1, flags=8)) == B.ERR_ARG
+    # variant flags only where they mean something
+    assert call(hyper=B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1, flags=B.FLAG_TWOSUM_GROW)) == B.ERR_ARG      # option A
+    kahan_bad = B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1, flags=B.FLAG_DECAY_BY_GROW)
+    assert call(strategy=B.KAHAN, x_lo=dummy * 5, hyper=kahan_bad) == B.ERR_ARG
     assert call(x_hi=None) == B.ERR_NULL
     assert call(grad=None) == B.ERR_NULL
     assert call(strategy=B.LIGHT) == B.ERR_NULL                      # x_lo missing
