@@ -221,3 +221,19 @@ def adamw_fp64(theta, m, v, grad, *, lr, beta1, beta2, eps, weight_decay, step, 
                             ctypes.c_double(eps), ctypes.c_double(weight_decay), ctypes.c_uint32(flags),
                             ctypes.c_uint64(step), _p(delta))
     return delta
+
+
+def adamw_fp32_step(theta, master, m, v, grad, *, lr, beta1, beta2, eps, weight_decay, step, flags=0):
+    """Comparator option D (master = float32 array) / D^-MW (master = None), in place.
+
+    theta, grad: uint16 bfloat16 bit patterns; m, v, master: float32.  Returns the EDQ sums dict.
+    """
+    assert theta.dtype == np.uint16 and m.dtype == np.float32 and v.dtype == np.float32
+    assert master is None or master.dtype == np.float32
+    grad = _u16(grad)
+    sums = np.zeros(4, dtype=np.float64)
+    lib().oracle_adamw_fp32_step(_p(theta), _p(master), _p(m), _p(v), _p(grad), ctypes.c_uint64(theta.size),
+                                 ctypes.c_double(lr), ctypes.c_double(beta1), ctypes.c_double(beta2),
+                                 ctypes.c_double(eps), ctypes.c_double(weight_decay), ctypes.c_uint32(flags),
+                                 ctypes.c_uint64(step), _p(sums))
+    return dict(dot=float(sums[0]), sumsq=float(sums[1]), edq=float(sums[2]), lost=int(sums[3]))

@@ -436,6 +436,64 @@ void oracle_adamw_fp64(double* theta, double* m, double* v, const double* grad, 
     }
 }
 
+// ---- comparator: option D of Table 2 (bfloat16 parameter and gradient, float optimizer states,
+// float master weights) and D^-MW (Section 5.1: the same without master weights) -----------------
+// Standard mixed-precision AdamW: every operation below is one IEEE single-precision operation
+// (this file is compiled with contraction off), scalars are evaluated in double and cast to float
+// once (Appendix D, scalar rule).  master == NULL selects D^-MW: the update is added to the
+// bfloat16 parameter widened to float and the sum is rounded back to bfloat16.
+// EDQ (Eq. 2-3): intended update = the float update; effective update = change of the stored
+// parameter (the master weight for D, the bfloat16 parameter for D^-MW), summed in double.
+void oracle_adamw_fp32_step(uint16_t* theta, float* master, float* m, float* v, const uint16_t* grad, uint64_t n,
+                            double lr, double beta1, double beta2, double eps, double wd, uint32_t flags,
+                            uint64_t step, double* sums_out) {
+    const float b1 = static_cast<float>(beta1), c1 = static_cast<float>(1.0 - beta1);
+    const float b2 = static_cast<float>(beta2), c2 = static_cast<float>(1.0 - beta2);
+    const float bc1 = static_cast<float>(1.0 - std::pow(beta1, static_cast<double>(step)));
+    const float bc2 = static_cast<float>(1.0 - std::pow(beta2, static_cast<double>(step)));
+    const float neg_a = -static_cast<float>(lr), lam = static_cast<float>(wd), epsf = static_cast<float>(eps);
+    edq_sums tot{0.0, 0.0, 0};
+    for (uint64_t i = 0; i < n; ++i) {
+        const float g = static_cast<float>(widen(grad[i]));
+        const float m_new = b1 * m[i] + c1 * g;
+        const float gg = g * g;
+        const float v_new = b2 * v[i] + c2 * gg;
+        m[i] = m_new;
+        v[i] = v_new;
+        const float mhat = m_new / bc1;
+        const float vhat = v_new / bc2;
+        const float den = (flags & FLAG_EPS_INSIDE_SQRT) ? std::sqrt(vhat + epsf) : std::sqrt(vhat) + epsf;
+        const float w_old = master ? master[i] : static_cast<float>(widen(theta[i]));
+        const float r = mhat / den;
+        const float decay = lam * w_old;
+        const float u = r + decay;
+        const float delta = neg_a * u;
+        const float w_new = w_old + delta;
+        const uint16_t theta_new = round_to_bf16(static_cast<double>(w_new));
+        double eff;
+        bool unchanged;
+        if (master) {
+            master[i] = w_new;
+            eff = static_cast<double>(w_new) - static_cast<double>(w_old);
+            unchanged = (w_new == w_old);
+        } else {
+            eff = widen(theta_new) - widen(theta[i]);
+            unchanged = (widen(theta_new) == widen(theta[i]));
+        }
+        theta[i] = theta_new;
+        const double d = static_cast<double>(delta);
+        tot.dot += d * eff;
+        tot.sumsq += d * d;
+        if (d != 0.0 && unchanged) tot.lost += 1;
+    }
+    if (sums_out) {
+        sums_out[0] = tot.dot;
+        sums_out[1] = tot.sumsq;
+        sums_out[2] = tot.sumsq > 0.0 ? tot.dot / std::sqrt(tot.sumsq) : 0.0;
+        sums_out[3] = static_cast<double>(tot.lost);
+    }
+}
+
 int oracle_max_threads(void) {
 #ifdef _OPENMP
     return omp_get_max_threads();
