@@ -308,6 +308,53 @@ def run_size_sweep(args):
             torch.cuda.empty_cache()
 
 
+def run_strategy_sweep(args):
+    """All precision options, the comparators and the step variants on one flat 2^30-parameter tensor."""
+    import torch
+    from paper_2405_03637_b200 import binding as B
+    from paper_2405_03637_b200 import workloads as W
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(device)
+    peak, _ = measured_hbm_peak()
+    n = 1 << 30
+    x = W.flat_weights(n, 0, device)
+    z = lambda: torch.zeros_like(x)
+    xl, m, v, vl, g = z(), z(), z(), z(), W.flat_grads(n, 0, 1, device)
+    edq_dev = torch.zeros(64, dtype=torch.uint8, device=device)
+    ws = torch.empty(B.workspace_bytes(), dtype=torch.uint8, device=device)
+    stream = torch.cuda.current_stream()
+    cases = [("A plain bf16", B.BF16, 0, 14), ("B collage-light", B.LIGHT, 0, 18), ("C collage-plus", B.PLUS, 0, 22),
+             ("BF16-Kahan", B.KAHAN, 0, 18), ("B + TwoSum Grow", B.LIGHT, B.FLAG_TWOSUM_GROW, 18),
+             ("C + TwoSum Grow", B.PLUS, B.FLAG_TWOSUM_GROW, 22), ("C + decay by Grow", B.PLUS, B.FLAG_DECAY_BY_GROW, 22)]
+    def timed(call, bytes_per_param, name):
+        for t in range(1, 4):
+            call(t)
+        torch.cuda.synchronize()
+        iters = 40
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+        ev[0].record(stream)
+        for i in range(iters):
+            call(4 + i)
+            ev[i + 1].record(stream)
+        torch.cuda.synchronize()
+        ts = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(iters))
+        ms = ts[len(ts) // 2]
+        gbs = n * bytes_per_param / (ms * 1e-3) / 1e9
+        print(json.dumps({"step": name, "n": n, "ms_per_step": ms, "params_per_sec": n / (ms * 1e-3),
+                          "bytes_per_param": bytes_per_param, "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak}), flush=True)
+    for name, strategy, flags, bpp in cases:
+        h = B.make_hyper(**W.HYPERS, flags=flags, edq_out=edq_dev, workspace=ws)
+        a = (x, xl if strategy >= 1 else None, m, v, vl if strategy == 2 else None, g)
+        timed(lambda t: B.adamw_step(*a, n, h, t, strategy, stream), bpp, name)
+    del xl, vl, m, v
+    torch.cuda.empty_cache()
+    m32, v32 = torch.zeros(n, dtype=torch.float32, device=device), torch.zeros(n, dtype=torch.float32, device=device)
+    master = x.float()
+    h = B.make_hyper(**W.HYPERS, edq_out=edq_dev, workspace=ws)
+    timed(lambda t: B.adamw_step_fp32(x, master, m32, v32, g, n, h, t, stream), 28, "D fp32 states + fp32 master")
+    timed(lambda t: B.adamw_step_fp32(x, None, m32, v32, g, n, h, t, stream), 22, "D^-MW fp32 states, no master")
+
+
 def run_cpu_baseline(W, seconds=15.0, threads=None):
     """The oracle as it stands on this machine's cores, on a bounded slice of the same workload."""
     import numpy as np
@@ -375,10 +422,13 @@ def main():
     ap.add_argument("--skip-extras", action="store_true", help="no e2e and no CPU baseline (profiling runs)")
     ap.add_argument("--chunk-elems", type=int, default=0, help="chunk size of the multi-tensor plan (0 = library default)")
     ap.add_argument("--per-tensor", action="store_true", help="time the per-tensor EDQ variant of the step")
+    ap.add_argument("--strategy-sweep", action="store_true", help="time every option, comparator and variant on a flat tensor")
     ap.add_argument("--size-sweep", action="store_true", help="flat-tensor size sweep instead of the benchmark")
     args = ap.parse_args()
     if args.size_sweep:
         run_size_sweep(args)
+    elif args.strategy_sweep:
+        run_strategy_sweep(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

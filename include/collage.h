@@ -131,6 +131,22 @@ collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi,
                                     const void* grad, uint64_t n, const collage_hyper_t* hyper,
                                     uint64_t step, collage_strategy_t strategy, void* stream);
 
+/* Comparator of the paper's experiments: option D of Table 2 -- bfloat16 parameter and gradient,
+ * float (fp32) optimizer states and float master weights, 16 B/param -- and, with master == NULL,
+ * D^-MW of Section 5.1 (float optimizer states, no master weights, 12 B/param).  Standard
+ * mixed-precision AdamW in the operation order of Algorithm 2; every operation is one IEEE
+ * single-precision operation, scalars are evaluated in double and cast to float once.
+ *   theta : DEVICE bfloat16[n], written (D: theta = RN_bf16(master); D^-MW: read and written)
+ *   master: DEVICE float[n] or NULL;  m, v: DEVICE float[n];  grad: DEVICE bfloat16[n], read only
+ * EDQ (hyper->edq_out / workspace as for collage_adamw_step) measures the float update against the
+ * change of the stored parameter: the master weight for D, the bfloat16 parameter for D^-MW.
+ * HBM traffic 28 B/param (D) or 22 B/param (D^-MW) against 22 B/param of Collage-plus.
+ * Only COLLAGE_FLAG_EPS_INSIDE_SQRT is accepted in hyper->flags.
+ * Errors: ERR_NULL, ERR_ARG (step 0, hyper range, flags, float arrays not 4-byte aligned),
+ * ERR_ALIAS, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA. */
+collage_status_t collage_adamw_step_fp32(void* theta, void* master, void* m, void* v, const void* grad,
+                                         uint64_t n, const collage_hyper_t* hyper, uint64_t step, void* stream);
+
 /* The same step for state that lives in HOST memory (optimizer state kept off the device).
  * All six tensor pointers are HOST pointers (page-locked memory is needed for the copies to
  * overlap; pageable memory works, serialised by the runtime).  The arrays are streamed through

@@ -19,7 +19,7 @@ SCALAR_NAMES = ("b1", "c1", "b2", "c2", "b2h", "b2l", "bc1", "bc2", "a", "lam", 
 
 EXPORTS = (
     "collage_status_string", "collage_derive_scalars", "collage_workspace_bytes", "collage_adamw_step",
-    "collage_adamw_step_host",
+    "collage_adamw_step_host", "collage_adamw_step_fp32",
     "collage_plan_create", "collage_adamw_step_multi", "collage_plan_destroy", "collage_plan_num_elements",
     "collage_plan_num_chunks", "collage_plan_workspace_bytes", "collage_adamw_step_multi_per_tensor",
     "collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_grow",
@@ -74,6 +74,7 @@ def lib() -> ctypes.CDLL:
         L.collage_adamw_step.argtypes = [vp, vp, vp, vp, vp, vp, u64, ctypes.POINTER(Hyper), u64, i32, vp]
         L.collage_adamw_step_host.argtypes = [vp, vp, vp, vp, vp, vp, u64, ctypes.POINTER(Hyper), u64, i32, vp,
                                               ctypes.c_size_t, vp]
+        L.collage_adamw_step_fp32.argtypes = [vp, vp, vp, vp, vp, u64, ctypes.POINTER(Hyper), u64, vp]
         L.collage_plan_create.argtypes = [ctypes.POINTER(Tensor), i32, ctypes.c_uint32, ctypes.POINTER(vp)]
         L.collage_adamw_step_multi.argtypes = [vp, ctypes.POINTER(Hyper), u64, i32, vp]
         L.collage_plan_destroy.argtypes = [vp]
@@ -144,6 +145,12 @@ def adamw_step_host(x_hi, x_lo, m, v_hi, v_lo, grad, n, hyper: Hyper, step: int,
                                          ctypes.byref(hyper), step, strategy, _ptr(staging),
                                          staging.numel() * staging.element_size(), _ptr(stream)),
            "collage_adamw_step_host")
+
+
+def adamw_step_fp32(theta, master, m, v, grad, n, hyper: Hyper, step: int, stream=None):
+    """Comparator option D (master: float32 CUDA tensor) / D^-MW (master None); m, v float32, theta, grad bfloat16."""
+    _check(lib().collage_adamw_step_fp32(_ptr(theta), _ptr(master), _ptr(m), _ptr(v), _ptr(grad), n, ctypes.byref(hyper),
+                                         step, _ptr(stream)), "collage_adamw_step_fp32")
 
 
 def plan_create(tensors, chunk_elems: int = 0) -> int:

@@ -15,7 +15,7 @@ from pathlib import Path
 HERE = Path(__file__).resolve().parent
 CSRC = HERE / "csrc"
 LIB = HERE / "libcollage_b200.so"
-SOURCES = ["collage_step.cu", "collage_primitives.cu", "collage_edq_static.cu"]
+SOURCES = ["collage_step.cu", "collage_primitives.cu", "collage_edq_static.cu", "collage_fp32_master.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-fmad=false", "-ftz=false", "-prec-div=true", "-prec-sqrt=true",

@@ -451,6 +451,9 @@ static collage_status_t check_common(const collage_hyper_t* hyper, uint64_t step
 
 }  // namespace collage
 
+namespace collage {
+cudaError_t read_clear_fault32(unsigned int* out);
+}
 using namespace collage;
 
 struct collage_plan {
@@ -726,10 +729,11 @@ uint64_t collage_plan_num_chunks(const collage_plan_t* plan) { return plan ? pla
 
 collage_status_t collage_pipeline_fault(uint32_t* out_host) {
     if (!out_host) return COLLAGE_ERR_NULL;
-    unsigned int v = 0, zero = 0;
+    unsigned int v = 0, v32 = 0, zero = 0;
     if (cudaMemcpyFromSymbol(&v, g_pipeline_fault, sizeof v) != cudaSuccess) return COLLAGE_ERR_CUDA;
     if (v && cudaMemcpyToSymbol(g_pipeline_fault, &zero, sizeof zero) != cudaSuccess) return COLLAGE_ERR_CUDA;
-    *out_host = v;
+    if (read_clear_fault32(&v32) != cudaSuccess) return COLLAGE_ERR_CUDA;    // the float comparator's pipeline
+    *out_host = v ? v : v32;
     return COLLAGE_OK;
 }
 
