@@ -173,6 +173,8 @@ collage_status_t collage_adamw_step_host(void* x_hi, void* x_lo, void* m, void* 
  * Tensors with n == 0 are skipped.  The plan records which pointers were NULL; a step whose
  * strategy needs a missing component fails with ERR_NULL.  EDQ is over all tensors (Eq. 3
  * with theta the concatenation).
+ * A plan belongs to the device that was current at creation; stepping it with another device
+ * current is ERR_ARG.
  * Errors: ERR_NULL, ERR_ARG (num < 0, chunk_elems not a multiple of 2048, more than 2^32-1
  * chunks), ERR_ALIAS (any two arrays of the plan overlap), ERR_CUDA. */
 collage_status_t collage_plan_create(const collage_tensor_t* tensors, int num, uint32_t chunk_elems,

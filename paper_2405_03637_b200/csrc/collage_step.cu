@@ -471,6 +471,12 @@ struct collage_plan {
     int device = 0;
 };
 
+// a plan's tables live on the device that was current when it was created
+static bool plan_on_current_device(const collage_plan* plan) {
+    int device = -1;
+    return plan->num_tensors == 0 || (cudaGetDevice(&device) == cudaSuccess && device == plan->device);
+}
+
 extern "C" {
 
 const char* collage_status_string(collage_status_t status) {
@@ -640,6 +646,7 @@ collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const coll
     DeviceInfo dev;
     st = current_device(&dev);
     if (st != COLLAGE_OK) return st;
+    if (!plan_on_current_device(plan)) return COLLAGE_ERR_ARG;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
     StepParams p{};
@@ -687,6 +694,7 @@ collage_status_t collage_adamw_step_multi_per_tensor(const collage_plan_t* plan,
     DeviceInfo dev;
     st = current_device(&dev);
     if (st != COLLAGE_OK) return st;
+    if (!plan_on_current_device(plan)) return COLLAGE_ERR_ARG;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
     StepParams p{};

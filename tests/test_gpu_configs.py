@@ -189,3 +189,42 @@ def test_size_sweep_powers_of_four(strategy):
                 if st[k] is not None:
                     assert_same_bits(W.bits(d[k]), st[k], f"n=4^{p} step {t} {k}")
             edq_close(e.read(), want)
+
+
+def test_effective_descent_quality_orders_the_precision_strategies():
+    # Figure 3 (right) on synthetic data: share of the intended update that reaches the stored parameter,
+    # EDQ / ||update||, with config-0 distributions (updates around half an ulp of the parameters).  Plain
+    # bfloat16 loses part of every step, Kahan recovers it with a delay, the expansion-based options and
+    # fp32 master weights apply it all.
+    dev = torch.device("cuda")
+    n, hyp, steps = 1 << 22, W.HYPERS, 40
+    theta = W.flat_weights(n, 0, dev)
+    e = EdqBuffers()
+    quality = {}
+    for name, strategy in (("A", B.BF16), ("Kahan", B.KAHAN), ("B", B.LIGHT), ("C", B.PLUS)):
+        z = lambda: torch.zeros_like(theta)
+        d = dict(x_hi=theta.clone(), x_lo=z() if strategy else None, m=z(), v_hi=z(), v_lo=z() if strategy == 2 else None)
+        q = []
+        for t in range(1, steps + 1):
+            g = W.flat_grads(n, 0, t, dev)
+            B.adamw_step(d["x_hi"], d["x_lo"], d["m"], d["v_hi"], d["v_lo"], g, n, e.hyper(hyp), t, strategy)
+            torch.cuda.synchronize()
+            r = e.read()
+            q.append(r["edq"] / np.sqrt(r["sumsq"]))
+        quality[name] = q
+    master, m32, v32, th = theta.float(), torch.zeros(n, device=dev), torch.zeros(n, device=dev), theta.clone()
+    q = []
+    for t in range(1, steps + 1):
+        g = W.flat_grads(n, 0, t, dev)
+        B.adamw_step_fp32(th, master, m32, v32, g, n, e.hyper(hyp), t)
+        torch.cuda.synchronize()
+        r = e.read()
+        q.append(r["edq"] / np.sqrt(r["sumsq"]))
+    quality["D"] = q
+    mean = {k: float(np.mean(v)) for k, v in quality.items()}
+    print({k: (round(v[0], 4), round(v[-1], 4), round(mean[k], 4)) for k, v in quality.items()})
+    for k in ("B", "C", "D"):
+        assert min(quality[k]) > 0.995                               # the whole update arrives
+    assert mean["A"] < 0.95 * mean["B"]                              # plain bfloat16 loses a visible share
+    assert quality["Kahan"][0] == quality["A"][0]                    # first step: no compensation yet
+    assert mean["A"] < mean["Kahan"] <= 1.05                         # later steps deliver what earlier ones lost
