@@ -135,7 +135,9 @@ def run_collage(args):
         raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
-    if world > 1:
+    # under torchrun (any world size, 1 included) the ranks talk over NCCL; a bare `python bench.py` does not
+    use_dist = world > 1 or ("RANK" in os.environ and "MASTER_ADDR" in os.environ)
+    if use_dist:
         dist.init_process_group("nccl", device_id=device)
     B.lib()                                             # fail loudly if the CUDA library is missing
 
@@ -157,12 +159,12 @@ def run_collage(args):
             B.adamw_step_multi_per_tensor(plan, B.make_hyper(**hyp, edq_out=edq_dev), t, STRATEGY, per, len(rows), cws, stream)
         else:
             B.adamw_step_multi(plan, B.make_hyper(**hyp, edq_out=edq_dev, workspace=ws), t, STRATEGY, stream)
-        if world > 1:                                   # EDQ is global: sum the partial sums over ranks
+        if use_dist:                                    # EDQ is global: sum the partial sums over ranks
             dist.all_reduce(edq_sums)
             dist.all_reduce(edq_lost)
 
     def barrier():
-        if world > 1:
+        if use_dist:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -181,12 +183,12 @@ def run_collage(args):
         barrier()
     total_ms = ev[0].elapsed_time(ev[-1])
     per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    if world > 1:
+    if use_dist:
         tmax = torch.tensor([total_ms], dtype=torch.float64, device=device)
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         total_ms = float(tmax.item())
     edq = B.read_edq(edq_dev)
-    if world > 1:
+    if use_dist:
         edq["edq"] = edq["dot"] / edq["sumsq"] ** 0.5 if edq["sumsq"] > 0 else 0.0
 
     ms_per_step = total_ms / args.steps
@@ -199,7 +201,8 @@ def run_collage(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "params_per_gpu": n, "tensors": len(rows), "strategy": "collage_plus",
+        "config": {"workload": WORKLOAD if args.layers == 32 else f"{WORKLOAD}_reduced_to_{args.layers}_layers",
+                   "params_per_gpu": n, "tensors": len(rows), "strategy": "collage_plus",
                    "state_bytes_per_param": 12, "hbm_bytes_per_param_per_step": BYTES_PER_PARAM[STRATEGY],
                    "edq": True, "l2": "state (80.9 GB per GPU) far exceeds the 126 MB L2; no flush needed",
                    "parallelism": f"dp{world} (each rank owns a full 7B-shaped shard; EDQ sums all-reduced)"},
@@ -216,7 +219,7 @@ def run_collage(args):
         out["cpu_baseline"] = run_cpu_baseline(W, seconds=args.cpu_seconds)
     elif rank == 0:
         out["e2e"] = None
-    if world > 1:
+    if use_dist:
         dist.destroy_process_group()
     if rank == 0:
         print(json.dumps(out))
