@@ -237,3 +237,16 @@ def adamw_fp32_step(theta, master, m, v, grad, *, lr, beta1, beta2, eps, weight_
                                  ctypes.c_double(eps), ctypes.c_double(weight_decay), ctypes.c_uint32(flags),
                                  ctypes.c_uint64(step), _p(sums))
     return dict(dot=float(sums[0]), sumsq=float(sums[1]), edq=float(sums[2]), lost=int(sums[3]))
+
+
+def adamw_fp32_register_step(x_hi, x_lo, m, v_hi, v_lo, grad, *, lr, beta1, beta2, eps, weight_decay, step, flags=0):
+    """Variant: Collage-plus storage, float arithmetic in registers, re-split on store.  In place; EDQ sums dict."""
+    for arr in (x_hi, x_lo, m, v_hi, v_lo):
+        assert arr.dtype == np.uint16 and arr.flags.c_contiguous
+    grad = _u16(grad)
+    sums = np.zeros(4, dtype=np.float64)
+    lib().oracle_adamw_fp32_register_step(_p(x_hi), _p(x_lo), _p(m), _p(v_hi), _p(v_lo), _p(grad),
+                                          ctypes.c_uint64(x_hi.size), ctypes.c_double(lr), ctypes.c_double(beta1),
+                                          ctypes.c_double(beta2), ctypes.c_double(eps), ctypes.c_double(weight_decay),
+                                          ctypes.c_uint32(flags), ctypes.c_uint64(step), _p(sums))
+    return dict(dot=float(sums[0]), sumsq=float(sums[1]), edq=float(sums[2]), lost=int(sums[3]))

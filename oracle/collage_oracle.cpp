@@ -494,6 +494,61 @@ void oracle_adamw_fp32_step(uint16_t* theta, float* master, float* m, float* v, 
     }
 }
 
+// ---- variant: float arithmetic in registers on the Collage-plus storage -------------------------
+// Not in the paper (its Algorithm 2 is strict bfloat16); a measuring stick for what the strict
+// arithmetic costs at equal memory traffic.  Storage is option C's: (theta, dtheta), m, (v, dv) in
+// bfloat16.  Each step widens to float (theta + dtheta and v + dv by one float addition), runs
+// AdamW exactly as the option-D comparator does (IEEE single operations, float scalars), and
+// splits the results back: hi = RN_bf16(x), lo = RN_bf16(x - hi).
+void oracle_adamw_fp32_register_step(uint16_t* x_hi, uint16_t* x_lo, uint16_t* m, uint16_t* v_hi, uint16_t* v_lo,
+                                     const uint16_t* grad, uint64_t n, double lr, double beta1, double beta2,
+                                     double eps, double wd, uint32_t flags, uint64_t step, double* sums_out) {
+    const float b1 = static_cast<float>(beta1), c1 = static_cast<float>(1.0 - beta1);
+    const float b2 = static_cast<float>(beta2), c2 = static_cast<float>(1.0 - beta2);
+    const float bc1 = static_cast<float>(1.0 - std::pow(beta1, static_cast<double>(step)));
+    const float bc2 = static_cast<float>(1.0 - std::pow(beta2, static_cast<double>(step)));
+    const float neg_a = -static_cast<float>(lr), lam = static_cast<float>(wd), epsf = static_cast<float>(eps);
+    auto f = [](uint16_t h) { return static_cast<float>(widen(h)); };
+    edq_sums tot{0.0, 0.0, 0};
+    for (uint64_t i = 0; i < n; ++i) {
+        const float g = f(grad[i]);
+        const float x = f(x_hi[i]) + f(x_lo[i]);
+        const float vv = f(v_hi[i]) + f(v_lo[i]);
+        const float m_new = b1 * f(m[i]) + c1 * g;
+        const float gg = g * g;
+        const float v_new = b2 * vv + c2 * gg;
+        const float mhat = m_new / bc1;
+        const float vhat = v_new / bc2;
+        const float den = (flags & FLAG_EPS_INSIDE_SQRT) ? std::sqrt(vhat + epsf) : std::sqrt(vhat) + epsf;
+        const float r = mhat / den;
+        const float decay = lam * x;
+        const float u = r + decay;
+        const float delta = neg_a * u;
+        const float x_new = x + delta;
+        const uint16_t th = round_to_bf16(static_cast<double>(x_new));
+        const uint16_t dth = round_to_bf16(static_cast<double>(x_new - f(th)));
+        const uint16_t vh = round_to_bf16(static_cast<double>(v_new));
+        const uint16_t vl = round_to_bf16(static_cast<double>(v_new - f(vh)));
+        const double eff = (widen(th) - widen(x_hi[i])) + (widen(dth) - widen(x_lo[i]));
+        const bool unchanged = widen(th) == widen(x_hi[i]) && widen(dth) == widen(x_lo[i]);
+        x_hi[i] = th;
+        x_lo[i] = dth;
+        m[i] = round_to_bf16(static_cast<double>(m_new));
+        v_hi[i] = vh;
+        v_lo[i] = vl;
+        const double d = static_cast<double>(delta);
+        tot.dot += d * eff;
+        tot.sumsq += d * d;
+        if (d != 0.0 && unchanged) tot.lost += 1;
+    }
+    if (sums_out) {
+        sums_out[0] = tot.dot;
+        sums_out[1] = tot.sumsq;
+        sums_out[2] = tot.sumsq > 0.0 ? tot.dot / std::sqrt(tot.sumsq) : 0.0;
+        sums_out[3] = static_cast<double>(tot.lost);
+    }
+}
+
 int oracle_max_threads(void) {
 #ifdef _OPENMP
     return omp_get_max_threads();

@@ -107,3 +107,67 @@ def test_no_master_weights_rounds_the_float_sum_to_bf16():
     gf = bits_to_f64(g)
     want = bits_to_f64(before) - 1e-4 * (gf / (np.abs(gf) + 1e-8) + 0.1 * bits_to_f64(before))
     assert np.mean(theta == oracle.round_to_bf16(want)) > 0.999      # all but float-vs-double near-ties
+
+
+# ---- variant: float arithmetic in registers on the Collage-plus storage ---------------------------
+
+def _pair_state(n, seed):
+    theta = W.bits(W.flat_weights(n, seed))
+    z = lambda: np.zeros(n, np.uint16)
+    return dict(x_hi=theta, x_lo=z(), m=z(), v_hi=z(), v_lo=z())
+
+
+def test_register_variant_stores_normalised_pairs_and_tracks_fp64_adamw():
+    n, T = 1 << 14, 50
+    hyp = dict(HYP, beta2=0.95)
+    st = _pair_state(n, 0)
+    strict = {k: v.copy() for k, v in st.items()}
+    th64 = bits_to_f64(st["x_hi"]).copy(); m64 = np.zeros(n); v64 = np.zeros(n)
+    moved = np.zeros(n)
+    for t in range(1, T + 1):
+        g = W.bits(W.flat_grads(n, 0, t))
+        s = oracle.adamw_fp32_register_step(st["x_hi"], st["x_lo"], st["m"], st["v_hi"], st["v_lo"], g, step=t, **hyp)
+        oracle.adamw_step(strict["x_hi"], strict["x_lo"], strict["m"], strict["v_hi"], strict["v_lo"], g, step=t,
+                          strategy=oracle.STRATEGY_PLUS, **hyp)
+        moved += np.abs(oracle.adamw_fp64(th64, m64, v64, bits_to_f64(g), step=t, want_delta=True, **hyp))
+        # the split is a normalised expansion (Def. 2.1): |lo| <= ulp(hi)/2, for theta and for v
+        from conftest import ulp_f64
+        assert np.all(np.abs(bits_to_f64(st["x_lo"])) <= ulp_f64(st["x_hi"]) / 2)
+        assert np.all(np.abs(bits_to_f64(st["v_lo"])) <= ulp_f64(st["v_hi"]) / 2)
+        assert s["lost"] <= n // 100                          # updates below the ~2^-17 resolution of the pair
+    held = bits_to_f64(st["x_hi"]) + bits_to_f64(st["x_lo"])
+    held_strict = bits_to_f64(strict["x_hi"]) + bits_to_f64(strict["x_lo"])
+    err, err_strict = np.abs(held - th64), np.abs(held_strict - th64)
+    # a bfloat16 pair resolves ~2^-16 of theta per step; m is stored in bfloat16 (2^-9 relative), which bounds
+    # how far the update can drift from the double one
+    assert np.all(err <= 0.01 * moved + T * 2.0 ** -16 * np.abs(th64))
+    # and float arithmetic in registers sits closer to the double trajectory than strict bfloat16 arithmetic
+    assert err.sum() < 0.5 * err_strict.sum()
+    vv = bits_to_f64(st["v_hi"]) + bits_to_f64(st["v_lo"])
+    assert np.all(np.abs(vv - v64) <= 2.0 ** -14 * v64 + 1e-30)
+
+
+def test_register_variant_matches_a_numpy_float32_evaluation():
+    n = 1 << 12
+    f = np.float32
+    hyp = dict(lr=3e-3, beta1=0.9, beta2=0.98, eps=1e-6, weight_decay=0.01)
+    st = _pair_state(n, 4)
+    ref = {k: v.copy() for k, v in st.items()}
+    w = lambda b: bits_to_f64(b).astype(f)
+    rn = lambda x: oracle.round_to_bf16(x.astype(np.float64))
+    for t in range(1, 6):
+        gb = W.bits(W.flat_grads(n, 4, t))
+        oracle.adamw_fp32_register_step(st["x_hi"], st["x_lo"], st["m"], st["v_hi"], st["v_lo"], gb, step=t, **hyp)
+        g = w(gb)
+        x = w(ref["x_hi"]) + w(ref["x_lo"])
+        vv = w(ref["v_hi"]) + w(ref["v_lo"])
+        m_new = f(hyp["beta1"]) * w(ref["m"]) + f(1.0 - hyp["beta1"]) * g
+        v_new = f(hyp["beta2"]) * vv + f(1.0 - hyp["beta2"]) * (g * g)
+        den = np.sqrt(v_new / f(1.0 - hyp["beta2"] ** t)) + f(hyp["eps"])
+        delta = f(-f(hyp["lr"])) * ((m_new / f(1.0 - hyp["beta1"] ** t)) / den + f(hyp["weight_decay"]) * x)
+        x_new = x + delta
+        ref["x_hi"] = rn(x_new); ref["x_lo"] = rn(x_new - w(ref["x_hi"]))
+        ref["m"] = rn(m_new)
+        ref["v_hi"] = rn(v_new); ref["v_lo"] = rn(v_new - w(ref["v_hi"]))
+        for k in st:
+            assert np.array_equal(st[k], ref[k]), (t, k)
