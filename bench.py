@@ -328,7 +328,8 @@ def run_strategy_sweep(args):
     stream = torch.cuda.current_stream()
     cases = [("A plain bf16", B.BF16, 0, 14), ("B collage-light", B.LIGHT, 0, 18), ("C collage-plus", B.PLUS, 0, 22),
              ("BF16-Kahan", B.KAHAN, 0, 18), ("B + TwoSum Grow", B.LIGHT, B.FLAG_TWOSUM_GROW, 18),
-             ("C + TwoSum Grow", B.PLUS, B.FLAG_TWOSUM_GROW, 22), ("C + decay by Grow", B.PLUS, B.FLAG_DECAY_BY_GROW, 22)]
+             ("C + TwoSum Grow", B.PLUS, B.FLAG_TWOSUM_GROW, 22), ("C + decay by Grow", B.PLUS, B.FLAG_DECAY_BY_GROW, 22),
+             ("C storage, fp32 arithmetic in registers", B.PLUS_FP32_REGISTERS, 0, 22)]
     def timed(call, bytes_per_param, name):
         for t in range(1, 4):
             call(t)
@@ -347,7 +348,7 @@ def run_strategy_sweep(args):
                           "bytes_per_param": bytes_per_param, "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak}), flush=True)
     for name, strategy, flags, bpp in cases:
         h = B.make_hyper(**W.HYPERS, flags=flags, edq_out=edq_dev, workspace=ws)
-        a = (x, xl if strategy >= 1 else None, m, v, vl if strategy == 2 else None, g)
+        a = (x, xl if strategy >= 1 else None, m, v, vl if strategy in (2, 4) else None, g)
         timed(lambda t: B.adamw_step(*a, n, h, t, strategy, stream), bpp, name)
     del xl, vl, m, v
     torch.cuda.empty_cache()

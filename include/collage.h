@@ -56,7 +56,12 @@ typedef enum {
      * at the parameter update (Appendix B): update' = update (+) c; theta' = theta (+) update';
      * c' = update' (-) (theta' (-) theta).  Same arrays as option B, x_lo holding c (10 B/param).
      * EDQ counts theta alone (Eq. 2 as printed). */
-    COLLAGE_KAHAN = 3
+    COLLAGE_KAHAN = 3,
+    /* A measuring stick outside the paper (its Algorithm 2 is strict bfloat16): option C's arrays and
+     * traffic, but each step widens theta+dtheta and v+dv to float, runs AdamW in IEEE single
+     * operations with float scalars, and splits the results back into normalised bfloat16 pairs
+     * (hi = RN(x), lo = RN(x - hi)).  Quantifies what the strict arithmetic costs in accuracy. */
+    COLLAGE_PLUS_FP32_REGISTERS = 4
 } collage_strategy_t;
 
 /* Algorithm 2 line 12 prints epsilon under the root; AdamW has it outside.  Default: outside. */
@@ -124,7 +129,8 @@ size_t collage_workspace_bytes(uint64_t n_total);
 /* One AdamW step over one flat tensor (Algorithm 2 lines 8-13, all n parameters, step t >= 1).
  *   x_hi, m, v_hi, grad : required.   x_lo : required iff strategy != COLLAGE_BF16 (delta-theta, or
  *   the Kahan compensation for COLLAGE_KAHAN), else must
- *   be NULL.   v_lo : required iff strategy == COLLAGE_PLUS, else must be NULL.
+ *   be NULL.   v_lo : required iff strategy is COLLAGE_PLUS or COLLAGE_PLUS_FP32_REGISTERS, else
+ *   must be NULL.
  * Errors: ERR_NULL, ERR_ARG (step 0, bad strategy, hyper range), ERR_ALIAS (overlapping
  * tensors), ERR_WORKSPACE (edq_out set, workspace too small), ERR_ARCH, ERR_CUDA. */
 collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi, void* v_lo,

@@ -105,21 +105,66 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
     uint32_t* dv = reinterpret_cast<uint32_t*>(&s.dv);
     const uint32_t* g = reinterpret_cast<const uint32_t*>(&s.g);
     EdqAcc acc = {0ull, 0ull, 0u};
+    if (STRATEGY == 4) {
+        // float arithmetic in registers: lane by lane, then the same EDQ terms on the stored pairs
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const bf2 th_old = th[j], dth_old = dth[j];
+            uint32_t lane[2][5];
+            float delta[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int sh = 16 * h;
+                lane[h][0] = (th[j] >> sh) & 0xFFFFu;
+                lane[h][1] = (dth[j] >> sh) & 0xFFFFu;
+                lane[h][2] = (m[j] >> sh) & 0xFFFFu;
+                lane[h][3] = (v[j] >> sh) & 0xFFFFu;
+                lane[h][4] = (dv[j] >> sh) & 0xFFFFu;
+                delta[h] = adamw_register_lane(lane[h][0], lane[h][1], lane[h][2], lane[h][3], lane[h][4],
+                                               (g[j] >> sh) & 0xFFFFu, k.f, k.flags);
+            }
+            th[j] = lane[0][0] | (lane[1][0] << 16);
+            dth[j] = lane[0][1] | (lane[1][1] << 16);
+            m[j] = lane[0][2] | (lane[1][2] << 16);
+            v[j] = lane[0][3] | (lane[1][3] << 16);
+            dv[j] = lane[0][4] | (lane[1][4] << 16);
+            if (EDQ) {
+                bf2 th_new = th[j], dth_new = dth[j];
+                const int lanes = valid - 2 * j;            // padded lanes hold zeros on input
+                if (lanes < 2) {
+                    const uint32_t mask = lanes == 1 ? 0x0000FFFFu : 0u;
+                    th_new &= mask;
+                    dth_new &= mask;
+                    if (lanes < 2) delta[1] = 0.0f;
+                    if (lanes < 1) delta[0] = 0.0f;
+                }
+                f32x2 d;
+                asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(delta[0]), "f"(delta[1]));
+                edq_pair_f<true>(acc, th_old, dth_old, th_new, dth_new, d);
+            }
+        }
+        if (EDQ) {
+            dot += static_cast<double>(edq_dot(acc));
+            sq += static_cast<double>(edq_sq(acc));
+            lost += acc.lost;
+        }
+        return;
+    }
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         ElemState e;
         e.th = th[j];
-        e.dth = STRATEGY >= 1 ? dth[j] : 0u;   // delta-theta (B, C) or the Kahan compensation
+        e.dth = stores_x_lo(STRATEGY) ? dth[j] : 0u;   // delta-theta (B, C) or the Kahan compensation
         e.m = m[j];
         e.v = v[j];
-        e.dv = STRATEGY == 2 ? dv[j] : 0u;
+        e.dv = stores_v_lo(STRATEGY) ? dv[j] : 0u;
         const bf2 th_old = e.th, dth_old = e.dth;
         const PairUpdate up = adamw_pair<STRATEGY, FAST, VARIANT>(e, g[j], k);
         th[j] = e.th;
         m[j] = e.m;
         v[j] = e.v;
-        if (STRATEGY >= 1) dth[j] = e.dth;
-        if (STRATEGY == 2) dv[j] = e.dv;
+        if (stores_x_lo(STRATEGY)) dth[j] = e.dth;
+        if (stores_v_lo(STRATEGY)) dv[j] = e.dv;
         if (EDQ) {
             bf2 th_new = e.th, dth_new = e.dth, delta = up.delta, decay = up.decay;
             if (valid < 8) {            // padded lanes hold zeros on input; keep them out of the sums
@@ -134,7 +179,7 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
             f32x2 d = widen2(delta);
             if (VARIANT && (k.flags & 4u)) d = add_f32x2(d, widen2(decay));
             // the stored parameter is the pair for options B and C, theta alone for A and Kahan
-            edq_pair_f<(STRATEGY == 1 || STRATEGY == 2)>(acc, th_old, dth_old, th_new, dth_new, d);
+            edq_pair_f<parameter_is_pair(STRATEGY)>(acc, th_old, dth_old, th_new, dth_new, d);
         }
     }
     if (EDQ) {
@@ -150,16 +195,16 @@ __device__ __forceinline__ void load_vec(Vec& s, const TensorRec& t, uint64_t of
     s.m = ld_stream(t.m + off);
     s.v = ld_stream(t.v_hi + off);
     s.g = ld_stream(t.grad + off);
-    if (STRATEGY >= 1) s.dth = ld_stream(t.x_lo + off);
-    if (STRATEGY == 2) s.dv = ld_stream(t.v_lo + off);
+    if (stores_x_lo(STRATEGY)) s.dth = ld_stream(t.x_lo + off);
+    if (stores_v_lo(STRATEGY)) s.dv = ld_stream(t.v_lo + off);
 }
 template <int STRATEGY>
 __device__ __forceinline__ void store_vec(const Vec& s, const TensorRec& t, uint64_t off) {
     st_stream(t.x_hi + off, s.th);
     st_stream(t.m + off, s.m);
     st_stream(t.v_hi + off, s.v);
-    if (STRATEGY >= 1) st_stream(t.x_lo + off, s.dth);
-    if (STRATEGY == 2) st_stream(t.v_lo + off, s.dv);
+    if (stores_x_lo(STRATEGY)) st_stream(t.x_lo + off, s.dth);
+    if (stores_v_lo(STRATEGY)) st_stream(t.v_lo + off, s.dv);
 }
 template <int STRATEGY>
 __device__ __forceinline__ void load_elems(Vec& s, const TensorRec& t, uint64_t off, int count) {
@@ -167,16 +212,16 @@ __device__ __forceinline__ void load_elems(Vec& s, const TensorRec& t, uint64_t 
     s.m = ld_elems(t.m + off, count);
     s.v = ld_elems(t.v_hi + off, count);
     s.g = ld_elems(t.grad + off, count);
-    if (STRATEGY >= 1) s.dth = ld_elems(t.x_lo + off, count);
-    if (STRATEGY == 2) s.dv = ld_elems(t.v_lo + off, count);
+    if (stores_x_lo(STRATEGY)) s.dth = ld_elems(t.x_lo + off, count);
+    if (stores_v_lo(STRATEGY)) s.dv = ld_elems(t.v_lo + off, count);
 }
 template <int STRATEGY>
 __device__ __forceinline__ void store_elems(const Vec& s, const TensorRec& t, uint64_t off, int count) {
     st_elems(t.x_hi + off, s.th, count);
     st_elems(t.m + off, s.m, count);
     st_elems(t.v_hi + off, s.v, count);
-    if (STRATEGY >= 1) st_elems(t.x_lo + off, s.dth, count);
-    if (STRATEGY == 2) st_elems(t.v_lo + off, s.dv, count);
+    if (stores_x_lo(STRATEGY)) st_elems(t.x_lo + off, s.dth, count);
+    if (stores_v_lo(STRATEGY)) st_elems(t.v_lo + off, s.dv, count);
 }
 
 }  // namespace collage
@@ -311,6 +356,18 @@ static collage_status_t make_scalars(const collage_hyper_t* hyper, uint64_t step
     k->lam = dup(s[9]);
     k->eps = dup(s[10]);
     k->flags = hyper->flags;
+    {   // float scalars of the register variant: each expression in double, one cast
+        const double t = static_cast<double>(step);
+        k->f.b1 = static_cast<float>(hyper->beta1);
+        k->f.c1 = static_cast<float>(1.0 - hyper->beta1);
+        k->f.b2 = static_cast<float>(hyper->beta2);
+        k->f.c2 = static_cast<float>(1.0 - hyper->beta2);
+        k->f.bc1 = static_cast<float>(1.0 - std::pow(hyper->beta1, t));
+        k->f.bc2 = static_cast<float>(1.0 - std::pow(hyper->beta2, t));
+        k->f.neg_a = -static_cast<float>(hyper->lr);
+        k->f.lam = static_cast<float>(hyper->weight_decay);
+        k->f.eps = static_cast<float>(hyper->eps);
+    }
     // the lean arithmetic chain of the kernel is valid for these ranges (every practical setting)
     const double bc1 = bf16_to_double(s[6]), bc2 = bf16_to_double(s[7]), eps = bf16_to_double(s[10]);
     k->fast = (bc1 >= 0x1p-100 && bc1 <= 1.0 && bc2 >= 0x1p-100 && bc2 <= 1.0 && eps >= 0x1p-54 && eps <= 0x1p60) ? 1u : 0u;
@@ -358,7 +415,9 @@ static cudaError_t dispatch_step2(const StepParams& p, int strategy, bool edq, i
         case 4: return launch_step<2, false, FLAT, FAST>(p, sm_count, stream, grid_out);
         case 5: return launch_step<2, true, FLAT, FAST>(p, sm_count, stream, grid_out);
         case 6: return launch_step<3, false, FLAT, FAST>(p, sm_count, stream, grid_out);
-        default: return launch_step<3, true, FLAT, FAST>(p, sm_count, stream, grid_out);
+        case 7: return launch_step<3, true, FLAT, FAST>(p, sm_count, stream, grid_out);
+        case 8: return launch_step<4, false, FLAT, false>(p, sm_count, stream, grid_out);   // no bfloat16 chain: FAST is moot
+        default: return launch_step<4, true, FLAT, false>(p, sm_count, stream, grid_out);
     }
 }
 // multi-tensor step with one EDQ record per chunk
@@ -372,7 +431,8 @@ static cudaError_t dispatch_step_per_chunk(const StepParams& p, int strategy, in
         case 4: return launch_step<2, true, false, false, true>(p, sm_count, stream, grid_out);
         case 5: return launch_step<2, true, false, true, true>(p, sm_count, stream, grid_out);
         case 6: return launch_step<3, true, false, false, true>(p, sm_count, stream, grid_out);
-        default: return launch_step<3, true, false, true, true>(p, sm_count, stream, grid_out);
+        case 7: return launch_step<3, true, false, true, true>(p, sm_count, stream, grid_out);
+        default: return launch_step<4, true, false, false, true>(p, sm_count, stream, grid_out);
     }
 }
 
@@ -434,14 +494,14 @@ static cudaError_t launch_flat(void* x_hi, void* x_lo, void* m, void* v_hi, void
 static collage_status_t check_common(const collage_hyper_t* hyper, uint64_t step, int strategy) {
     if (!hyper) return COLLAGE_ERR_NULL;
     if (step == 0) return COLLAGE_ERR_ARG;
-    if (strategy < COLLAGE_BF16 || strategy > COLLAGE_KAHAN) return COLLAGE_ERR_ARG;
+    if (strategy < COLLAGE_BF16 || strategy > COLLAGE_PLUS_FP32_REGISTERS) return COLLAGE_ERR_ARG;
     if (!hyper_in_range(hyper)) return COLLAGE_ERR_ARG;
     if (hyper->flags & ~(COLLAGE_FLAG_EPS_INSIDE_SQRT | COLLAGE_FLAG_TWOSUM_GROW | COLLAGE_FLAG_DECAY_BY_GROW))
         return COLLAGE_ERR_ARG;
     // TwoSum Grow needs a parameter pair (B, C); the Kahan comparator takes neither variant
     if ((hyper->flags & COLLAGE_FLAG_TWOSUM_GROW) && strategy != COLLAGE_LIGHT && strategy != COLLAGE_PLUS)
         return COLLAGE_ERR_ARG;
-    if ((hyper->flags & COLLAGE_FLAG_DECAY_BY_GROW) && strategy == COLLAGE_KAHAN) return COLLAGE_ERR_ARG;
+    if ((hyper->flags & COLLAGE_FLAG_DECAY_BY_GROW) && strategy >= COLLAGE_KAHAN) return COLLAGE_ERR_ARG;
     if (hyper->edq_out) {
         if (!hyper->workspace || hyper->workspace_bytes < kWorkspaceBytes) return COLLAGE_ERR_WORKSPACE;
         if (reinterpret_cast<uintptr_t>(hyper->workspace) & 15u) return COLLAGE_ERR_WORKSPACE;
@@ -520,7 +580,7 @@ collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi,
     if (st != COLLAGE_OK) return st;
     if (!x_hi || !m || !v_hi || !grad) return COLLAGE_ERR_NULL;
     if ((strategy >= COLLAGE_LIGHT) != (x_lo != nullptr)) return x_lo ? COLLAGE_ERR_ARG : COLLAGE_ERR_NULL;
-    if ((strategy == COLLAGE_PLUS) != (v_lo != nullptr)) return v_lo ? COLLAGE_ERR_ARG : COLLAGE_ERR_NULL;
+    if (stores_v_lo(strategy) != (v_lo != nullptr)) return v_lo ? COLLAGE_ERR_ARG : COLLAGE_ERR_NULL;
     if (n > (1ull << 62)) return COLLAGE_ERR_ARG;
     std::vector<ByteRange> ranges;
     for (const void* q : {static_cast<const void*>(x_hi), static_cast<const void*>(x_lo), static_cast<const void*>(m),
@@ -642,7 +702,7 @@ collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const coll
     collage_status_t st = check_common(hyper, step, strategy);
     if (st != COLLAGE_OK) return st;
     if (strategy >= COLLAGE_LIGHT && !plan->has_x_lo) return COLLAGE_ERR_NULL;
-    if (strategy == COLLAGE_PLUS && !plan->has_v_lo) return COLLAGE_ERR_NULL;
+    if (stores_v_lo(strategy) && !plan->has_v_lo) return COLLAGE_ERR_NULL;
     DeviceInfo dev;
     st = current_device(&dev);
     if (st != COLLAGE_OK) return st;
@@ -687,7 +747,7 @@ collage_status_t collage_adamw_step_multi_per_tensor(const collage_plan_t* plan,
     if (num != plan->num_given) return COLLAGE_ERR_ARG;
     if (h.flags & (COLLAGE_FLAG_TWOSUM_GROW | COLLAGE_FLAG_DECAY_BY_GROW)) return COLLAGE_ERR_ARG;   // not built
     if (strategy >= COLLAGE_LIGHT && !plan->has_x_lo) return COLLAGE_ERR_NULL;
-    if (strategy == COLLAGE_PLUS && !plan->has_v_lo) return COLLAGE_ERR_NULL;
+    if (stores_v_lo(strategy) && !plan->has_v_lo) return COLLAGE_ERR_NULL;
     if (!chunk_workspace || (reinterpret_cast<uintptr_t>(chunk_workspace) & 15u) ||
         chunk_workspace_bytes < collage_plan_workspace_bytes(plan))
         return COLLAGE_ERR_WORKSPACE;
@@ -786,7 +846,7 @@ collage_status_t collage_adamw_step_host(void* x_hi, void* x_lo, void* m, void* 
     if (st != COLLAGE_OK) return st;
     if (!x_hi || !m || !v_hi || !grad) return COLLAGE_ERR_NULL;
     if ((strategy >= COLLAGE_LIGHT) != (x_lo != nullptr)) return x_lo ? COLLAGE_ERR_ARG : COLLAGE_ERR_NULL;
-    if ((strategy == COLLAGE_PLUS) != (v_lo != nullptr)) return v_lo ? COLLAGE_ERR_ARG : COLLAGE_ERR_NULL;
+    if (stores_v_lo(strategy) != (v_lo != nullptr)) return v_lo ? COLLAGE_ERR_ARG : COLLAGE_ERR_NULL;
     if (n > (1ull << 62)) return COLLAGE_ERR_ARG;
     std::vector<ByteRange> ranges;
     for (const void* q : {static_cast<const void*>(x_hi), static_cast<const void*>(x_lo), static_cast<const void*>(m),

@@ -287,6 +287,11 @@ __device__ __forceinline__ bf2pair mcf_mul2(bf2 a1, bf2 a2, bf2 b1, bf2 b2) {
 
 // ------------------------------------------------------------ AdamW step ---
 
+// float scalars of the register variant (cast from double once, like the option-D comparator's)
+struct FloatScalars {
+    float b1, c1, b2, c2, bc1, bc2, neg_a, lam, eps;
+};
+
 // bfloat16 scalars of one step, each duplicated into both halves of a bf2 (Algorithm 2 line 1).
 struct StepScalars {
     bf2 b1, c1;        // RN(beta1), RN(1-beta1)
@@ -299,11 +304,20 @@ struct StepScalars {
     bf2 eps;           // RN(eps)
     uint32_t flags;    // bit 0: epsilon under the root; bit 1: TwoSum Grow; bit 2: decay by its own addition
     uint32_t fast;     // host-checked: 2^-100 <= bc1, bc2 <= 1 and 2^-54 <= eps <= 2^60
+    FloatScalars f;    // only read by the register variant (strategy 4)
 };
 
 struct ElemState {
     bf2 th, dth, m, v, dv;
 };
+
+// which arrays a strategy stores: 0 = A, 1 = B, 2 = C, 3 = BF16-Kahan, 4 = float arithmetic in
+// registers on option C's storage
+__host__ __device__ constexpr bool stores_x_lo(int strategy) { return strategy >= 1; }
+__host__ __device__ constexpr bool stores_v_lo(int strategy) { return strategy == 2 || strategy == 4; }
+// the stored parameter is the pair (theta, dtheta): B, C and the register variant
+__host__ __device__ constexpr bool parameter_is_pair(int strategy) { return strategy == 1 || strategy == 2 || strategy == 4; }
+
 
 // Algorithm 2 lines 10-12 for two parameters: the update delta from m, v (first component) and theta.
 //
@@ -413,5 +427,35 @@ __device__ __forceinline__ void edq_pair(EdqAcc& acc, bf2 th_old, bf2 dth_old, b
 }
 __device__ __forceinline__ float edq_dot(const EdqAcc& a) { return __fadd_rn(lo_of(a.dot), hi_of(a.dot)); }
 __device__ __forceinline__ float edq_sq(const EdqAcc& a) { return __fadd_rn(lo_of(a.sq), hi_of(a.sq)); }
+
+// ---- variant: float arithmetic in registers on option C's storage (strategy 4) -----------------
+// One lane: widen, AdamW in IEEE single operations (the option-D comparator's order), split back
+// into normalised bfloat16 pairs.  Returns the float update; the lane's five values are updated.
+__device__ __forceinline__ uint32_t bf16_bits_rn(float x) {
+    uint16_t h;
+    asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(x));
+    return h;
+}
+__device__ __forceinline__ float adamw_register_lane(uint32_t& th, uint32_t& dth, uint32_t& m, uint32_t& v, uint32_t& dv,
+                                                     uint32_t g16, const FloatScalars& k, uint32_t flags) {
+    auto w = [](uint32_t h) { return __uint_as_float(h << 16); };
+    const float g = w(g16);
+    const float x = __fadd_rn(w(th), w(dth));
+    const float vv = __fadd_rn(w(v), w(dv));
+    const float m_new = __fadd_rn(__fmul_rn(k.b1, w(m)), __fmul_rn(k.c1, g));
+    const float v_new = __fadd_rn(__fmul_rn(k.b2, vv), __fmul_rn(k.c2, __fmul_rn(g, g)));
+    const float mhat = __fdiv_rn(m_new, k.bc1);
+    const float vhat = __fdiv_rn(v_new, k.bc2);
+    const float den = (flags & 1u) ? __fsqrt_rn(__fadd_rn(vhat, k.eps)) : __fadd_rn(__fsqrt_rn(vhat), k.eps);
+    const float u = __fadd_rn(__fdiv_rn(mhat, den), __fmul_rn(k.lam, x));
+    const float delta = __fmul_rn(k.neg_a, u);
+    const float x_new = __fadd_rn(x, delta);
+    th = bf16_bits_rn(x_new);
+    dth = bf16_bits_rn(__fsub_rn(x_new, w(th)));
+    m = bf16_bits_rn(m_new);
+    v = bf16_bits_rn(v_new);
+    dv = bf16_bits_rn(__fsub_rn(v_new, w(v)));
+    return delta;
+}
 
 }  // namespace collage

@@ -79,7 +79,7 @@ __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.a
 // Number of state arrays read / written per option
 template <int STRATEGY>
 struct ArrayCount {
-    static constexpr int kIn = 4 + (STRATEGY >= 1 ? 1 : 0) + (STRATEGY == 2 ? 1 : 0);
+    static constexpr int kIn = 4 + (stores_x_lo(STRATEGY) ? 1 : 0) + (stores_v_lo(STRATEGY) ? 1 : 0);
     static constexpr int kOut = kIn - 1;   // everything but the gradient
 };
 
@@ -90,8 +90,8 @@ __device__ __forceinline__ void tile_pointers(const TensorRec& t, uint64_t off, 
     out[a++] = t.x_hi + off;
     out[a++] = t.m + off;
     out[a++] = t.v_hi + off;
-    if (STRATEGY >= 1) out[a++] = t.x_lo + off;
-    if (STRATEGY == 2) out[a++] = t.v_lo + off;
+    if (stores_x_lo(STRATEGY)) out[a++] = t.x_lo + off;
+    if (stores_v_lo(STRATEGY)) out[a++] = t.v_lo + off;
     g = t.grad + off;
 }
 
@@ -240,16 +240,16 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                         v.th = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
                         v.m = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
                         v.v = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
-                        if (STRATEGY >= 1) v.dth = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
-                        if (STRATEGY == 2) v.dv = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
+                        if (stores_x_lo(STRATEGY)) v.dth = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
+                        if (stores_v_lo(STRATEGY)) v.dv = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
                         v.g = *reinterpret_cast<const uint4*>(&sm.data[s][a][e]);
                         compute_vec<STRATEGY, EDQ, FAST, VARIANT>(v, k, 8, dot, sq, lost);
                         a = 0;
                         *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.th;
                         *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.m;
                         *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.v;
-                        if (STRATEGY >= 1) *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.dth;
-                        if (STRATEGY == 2) *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.dv;
+                        if (stores_x_lo(STRATEGY)) *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.dth;
+                        if (stores_v_lo(STRATEGY)) *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.dv;
                     }
                     pipe::fence_async_smem();      // shared-memory writes must be visible to the bulk store
                 } else {

@@ -75,7 +75,7 @@ def test_argument_errors_are_reported_before_any_cuda_call(L):
                                              kw.get("strategy", B.BF16), None)
     assert L.collage_adamw_step(dummy, None, dummy, dummy, None, dummy, 16, None, 1, 0, None) == B.ERR_NULL
     assert call(step=0) == B.ERR_ARG
-    assert call(strategy=4) == B.ERR_ARG
+    assert call(strategy=5) == B.ERR_ARG
     assert call(strategy=B.KAHAN) == B.ERR_NULL                      # the compensation array is missing
     assert call(strategy=-1) == B.ERR_ARG
     for bad in (dict(lr=-1.0), dict(beta1=1.0), dict(beta2=1.5), dict(eps=float("nan")), dict(weight_decay=float("inf"))):

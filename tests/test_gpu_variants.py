@@ -90,3 +90,27 @@ def test_flag_combinations_that_mean_nothing_are_rejected():
     with pytest.raises(B.CollageError) as err:
         B.adamw_step(a[0], a[4], a[1], a[2], None, a[3], 64, B.make_hyper(**W.HYPERS, flags=B.FLAG_TWOSUM_GROW), 1, B.KAHAN)
     assert err.value.status == B.ERR_ARG
+
+
+@pytest.mark.parametrize("n,misalign,flags", [(1 << 20, 0, 0), (100_003, 0, 1), (4097, 3, 0), (9, 0, 0)])
+def test_float_arithmetic_in_registers_variant_bitwise(n, misalign, flags):
+    # option C's storage, float arithmetic, results split back into bfloat16 pairs
+    hyp = dict(W.HYPERS, beta2=0.98)
+    theta = W.bits(W.flat_weights(n, 90))
+    z = lambda: np.zeros(n, np.uint16)
+    st = dict(x_hi=theta.copy(), x_lo=z(), m=z(), v_hi=z(), v_lo=z())
+    dev = {k: Guarded(v, misalign) for k, v in st.items()}
+    e = EdqBuffers()
+    for t in (1, 2, 3, 4):
+        g = W.bits(W.flat_grads(n, 91, t))
+        G = Guarded(g, misalign)
+        B.adamw_step(dev["x_hi"].t, dev["x_lo"].t, dev["m"].t, dev["v_hi"].t, dev["v_lo"].t, G.t, n,
+                     e.hyper(hyp, flags), t, B.PLUS_FP32_REGISTERS)
+        torch.cuda.synchronize()
+        want = oracle.adamw_fp32_register_step(st["x_hi"], st["x_lo"], st["m"], st["v_hi"], st["v_lo"], g, step=t,
+                                               flags=flags, **hyp)
+        for k in KEYS:
+            assert_same_bits(dev[k].bits(), st[k], f"register variant step {t} {k}")
+            assert dev[k].guards_intact()
+        edq_close(e.read(), want)
+    assert B.pipeline_fault() == 0
