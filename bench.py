@@ -150,6 +150,13 @@ def run_collage(args):
     edq_lost = edq_dev[32:40].view(torch.int64)         # lost-update count
     stream = torch.cuda.current_stream()
 
+    if args.replicas:                                   # variant: theta also written to R replicas by the step kernel
+        rep_buffers = [torch.empty(n, dtype=torch.bfloat16, device=device) for _ in range(args.replicas)]
+        offs, off = [], 0
+        for r in rows:
+            offs.append(off)
+            off += r[6]
+        B.plan_set_replicas(plan, [[buf[o:o + r[6]] for o, r in zip(offs, rows)] for buf in rep_buffers])
     if args.per_tensor:                                 # variant: EDQ kept per tensor (three launches per step)
         per = torch.zeros(len(rows) * 40, dtype=torch.uint8, device=device)
         cws = torch.empty(B.plan_workspace_bytes(plan), dtype=torch.uint8, device=device)
@@ -204,7 +211,7 @@ def run_collage(args):
         "config": {"workload": WORKLOAD if args.layers == 32 else f"{WORKLOAD}_reduced_to_{args.layers}_layers",
                    "params_per_gpu": n, "tensors": len(rows), "strategy": "collage_plus",
                    "state_bytes_per_param": 12, "hbm_bytes_per_param_per_step": BYTES_PER_PARAM[STRATEGY],
-                   "edq": True, "l2": "state (80.9 GB per GPU) far exceeds the 126 MB L2; no flush needed",
+                   "edq": True, "theta_replicas": args.replicas, "l2": "state (80.9 GB per GPU) far exceeds the 126 MB L2; no flush needed",
                    "parallelism": f"dp{world} (each rank owns a full 7B-shaped shard; EDQ sums all-reduced)"},
         "gpu_launches": (3 if args.per_tensor else 2) * args.steps,
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -425,6 +432,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
     ap.add_argument("--skip-extras", action="store_true", help="no e2e and no CPU baseline (profiling runs)")
     ap.add_argument("--chunk-elems", type=int, default=0, help="chunk size of the multi-tensor plan (0 = library default)")
+    ap.add_argument("--replicas", type=int, default=0, help="also write theta to this many replica buffers (same GPU)")
     ap.add_argument("--per-tensor", action="store_true", help="time the per-tensor EDQ variant of the step")
     ap.add_argument("--strategy-sweep", action="store_true", help="time every option, comparator and variant on a flat tensor")
     ap.add_argument("--size-sweep", action="store_true", help="flat-tensor size sweep instead of the benchmark")

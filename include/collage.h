@@ -189,6 +189,25 @@ collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const coll
                                           uint64_t step, collage_strategy_t strategy, void* stream);
 collage_status_t collage_plan_destroy(collage_plan_t* plan);
 
+/* Replicas of the parameter (sharded optimizer state: each GPU steps its own slice of the
+ * parameters, every GPU needs all of theta for the next forward pass).  After this call every
+ * step of the plan also writes the updated first component theta of tensor i to each replica,
+ * tile by tile from inside the step kernel (the same bulk stores that write theta home), so the
+ * gather costs no extra kernel and overlaps the step.  The paper describes no collective; this is
+ * the one exchange its optimizer step would need (2 B/param per replica).
+ *   replicas : HOST array of num_replicas * num DEVICE pointers, replica r of tensors[i] at
+ *              replicas[r * num + i], `num` as given to collage_plan_create; each points to
+ *              tensors[i].n bfloat16 values in this GPU's memory or in a peer GPU's memory mapped
+ *              into this process (peer access enabled), and must have the same address modulo 16
+ *              as tensors[i].x_hi.  Entries of empty tensors are ignored.  num_replicas <= 15;
+ *              0 removes the replicas.
+ * The call synchronises the device and allocates a small table: do it once, outside the step loop.
+ * A replica holds the new theta once the step's kernel has finished; readers on other GPUs need
+ * their own ordering with that (an event, a barrier).  Plain bulk stores only, no multicast.
+ * Errors: ERR_NULL, ERR_ARG (count, alignment, wrong device), ERR_ALIAS (a replica overlaps an
+ * array of the plan or another replica), ERR_CUDA. */
+collage_status_t collage_plan_set_replicas(collage_plan_t* plan, const void* const* replicas, int num_replicas);
+
 /* The multi-tensor step with EDQ kept per tensor (Eq. 2-3 evaluated on each parameter tensor of the
  * plan separately; the lost-update count of Def. 3.2 per tensor gives the imprecision percentage of
  * Figure 3, left).  Same state update as collage_adamw_step_multi, bit for bit.

@@ -21,7 +21,7 @@ EXPORTS = (
     "collage_status_string", "collage_derive_scalars", "collage_workspace_bytes", "collage_adamw_step",
     "collage_adamw_step_host", "collage_adamw_step_fp32",
     "collage_plan_create", "collage_adamw_step_multi", "collage_plan_destroy", "collage_plan_num_elements",
-    "collage_plan_num_chunks", "collage_plan_workspace_bytes", "collage_adamw_step_multi_per_tensor",
+    "collage_plan_num_chunks", "collage_plan_set_replicas", "collage_plan_workspace_bytes", "collage_adamw_step_multi_per_tensor",
     "collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_grow",
     "collage_scaling", "collage_mul", "collage_renormalize", "collage_rounded_op", "collage_edq",
     "collage_selftest", "collage_pipeline_fault", "collage_edq_static",
@@ -82,6 +82,7 @@ def lib() -> ctypes.CDLL:
         L.collage_plan_num_elements.argtypes = [vp]
         L.collage_plan_num_chunks.restype = u64
         L.collage_plan_num_chunks.argtypes = [vp]
+        L.collage_plan_set_replicas.argtypes = [vp, ctypes.POINTER(vp), i32]
         L.collage_plan_workspace_bytes.restype = ctypes.c_size_t
         L.collage_plan_workspace_bytes.argtypes = [vp]
         L.collage_adamw_step_multi_per_tensor.argtypes = [vp, ctypes.POINTER(Hyper), u64, i32, vp, i32, vp,
@@ -166,6 +167,13 @@ def plan_create(tensors, chunk_elems: int = 0) -> int:
 def adamw_step_multi(plan: int, hyper: Hyper, step: int, strategy: int, stream=None):
     _check(lib().collage_adamw_step_multi(plan, ctypes.byref(hyper), step, strategy, _ptr(stream)),
            "collage_adamw_step_multi")
+
+
+def plan_set_replicas(plan: int, replicas):
+    """replicas: list (one per replica) of lists (one per tensor of the plan, None for empty tensors) of tensors/addresses."""
+    flat = [(_ptr(t) or 0) for rep in replicas for t in rep]
+    arr = (ctypes.c_void_p * max(len(flat), 1))(*flat)
+    _check(lib().collage_plan_set_replicas(plan, arr, len(replicas)), "collage_plan_set_replicas")
 
 
 def plan_workspace_bytes(plan: int) -> int:

@@ -69,6 +69,9 @@ struct StepParams {
     StepScalars k;
     EdqPartial* partials;       // one per block, or nullptr
     EdqPartial* chunk_partials; // one per chunk (per-tensor EDQ), or nullptr
+    const uint64_t* replica_bases;  // [num_replicas][num_plan_tensors] base addresses of theta replicas, or nullptr
+    int num_replicas;
+    int num_plan_tensors;
 };
 
 // ---- 16-byte streaming accesses for tiles that bypass the copy pipeline ---------------------
@@ -523,6 +526,10 @@ struct collage_plan {
     uint64_t* d_sizes = nullptr;         // per non-empty tensor
     uint32_t* d_orig_index = nullptr;    // position of the tensor in the caller's array
     int num_given = 0;                   // length of the caller's array
+    uint64_t* d_replica_bases = nullptr; // [num_replicas][num_tensors] (non-empty tensors only)
+    int num_replicas = 0;
+    std::vector<ByteRange> ranges;       // byte ranges of every array of the plan (overlap checks)
+    std::vector<collage_tensor_t> given; // the caller's array, as given
     uint64_t num_chunks = 0;
     uint64_t num_elements = 0;
     uint32_t chunk_elems = 0;
@@ -660,6 +667,8 @@ collage_status_t collage_plan_create(const collage_tensor_t* tensors, int num, u
 
     collage_plan* plan = new collage_plan;
     plan->num_given = num;
+    plan->ranges = ranges;
+    plan->given.assign(tensors, tensors + num);
     plan->num_chunks = chunks.size();
     plan->num_elements = total;
     plan->chunk_elems = chunk_elems;
@@ -717,6 +726,9 @@ collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const coll
     p.num_chunks = plan->num_chunks;
     p.chunk_elems = plan->chunk_elems;
     p.partials = static_cast<EdqPartial*>(hyper->workspace);
+    p.replica_bases = plan->d_replica_bases;
+    p.num_replicas = plan->num_replicas;
+    p.num_plan_tensors = plan->num_tensors;
     const bool edq = hyper->edq_out != nullptr;
     int grid = 0;
     if (plan->num_chunks > 0) {
@@ -726,6 +738,41 @@ collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const coll
         launch_edq_finalize(p.partials, grid, plan->num_elements, static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
         if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
+    return COLLAGE_OK;
+}
+
+collage_status_t collage_plan_set_replicas(collage_plan_t* plan, const void* const* replicas, int num_replicas) {
+    if (!plan) return COLLAGE_ERR_NULL;
+    if (num_replicas < 0 || num_replicas > 15) return COLLAGE_ERR_ARG;
+    if (num_replicas > 0 && !replicas) return COLLAGE_ERR_NULL;
+    if (!plan_on_current_device(plan)) return COLLAGE_ERR_ARG;
+    std::vector<uint64_t> bases;
+    std::vector<ByteRange> ranges = plan->ranges;
+    for (int r = 0; r < num_replicas; ++r) {
+        for (int i = 0; i < plan->num_given; ++i) {
+            const collage_tensor_t& t = plan->given[i];
+            if (t.n == 0) continue;
+            const void* q = replicas[static_cast<size_t>(r) * plan->num_given + i];
+            if (!q) return COLLAGE_ERR_NULL;
+            // a replica must sit like its tensor relative to 16-byte boundaries: tiles are copied whole
+            if ((reinterpret_cast<uintptr_t>(q) & 15u) != (reinterpret_cast<uintptr_t>(t.x_hi) & 15u)) return COLLAGE_ERR_ARG;
+            push_range(ranges, q, t.n);
+            bases.push_back(reinterpret_cast<uint64_t>(q));
+        }
+    }
+    if (any_overlap(ranges)) return COLLAGE_ERR_ALIAS;
+    uint64_t* d = nullptr;
+    if (!bases.empty()) {
+        if (cudaMalloc(&d, bases.size() * sizeof(uint64_t)) != cudaSuccess) return COLLAGE_ERR_CUDA;
+        if (cudaMemcpy(d, bases.data(), bases.size() * sizeof(uint64_t), cudaMemcpyHostToDevice) != cudaSuccess) {
+            cudaFree(d);
+            return COLLAGE_ERR_CUDA;
+        }
+    }
+    if (cudaDeviceSynchronize() != cudaSuccess) return COLLAGE_ERR_CUDA;   // no step may still read the old table
+    cudaFree(plan->d_replica_bases);
+    plan->d_replica_bases = d;
+    plan->num_replicas = bases.empty() ? 0 : num_replicas;
     return COLLAGE_OK;
 }
 
@@ -765,6 +812,9 @@ collage_status_t collage_adamw_step_multi_per_tensor(const collage_plan_t* plan,
     p.num_chunks = plan->num_chunks;
     p.chunk_elems = plan->chunk_elems;
     p.chunk_partials = static_cast<EdqPartial*>(chunk_workspace);
+    p.replica_bases = plan->d_replica_bases;
+    p.num_replicas = plan->num_replicas;
+    p.num_plan_tensors = plan->num_tensors;
     if (num > 0 && cudaMemsetAsync(per_tensor_out_dev, 0, static_cast<size_t>(num) * sizeof(collage_edq_t), cs) != cudaSuccess)
         return COLLAGE_ERR_CUDA;
     if (plan->num_chunks > 0) {
@@ -788,6 +838,7 @@ collage_status_t collage_plan_destroy(collage_plan_t* plan) {
     ok = (cudaFree(plan->d_first_chunk) == cudaSuccess) && ok;
     ok = (cudaFree(plan->d_sizes) == cudaSuccess) && ok;
     ok = (cudaFree(plan->d_orig_index) == cudaSuccess) && ok;
+    ok = (cudaFree(plan->d_replica_bases) == cudaSuccess) && ok;
     delete plan;
     return ok ? COLLAGE_OK : COLLAGE_ERR_CUDA;
 }

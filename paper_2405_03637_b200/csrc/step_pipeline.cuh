@@ -95,6 +95,11 @@ __device__ __forceinline__ void tile_pointers(const TensorRec& t, uint64_t off, 
     g = t.grad + off;
 }
 
+// address of element `elem` of tensor `tensor` in replica r (a plan-wide table of base addresses)
+__device__ __forceinline__ uint16_t* replica_ptr(const StepParams& p, int r, uint32_t tensor, uint64_t elem) {
+    return reinterpret_cast<uint16_t*>(p.replica_bases[static_cast<uint64_t>(r) * p.num_plan_tensors + tensor]) + elem;
+}
+
 template <int CONSUMERS, int VPT, int STAGES, int STRATEGY>
 struct PipeSmem {
     static constexpr int kTile = CONSUMERS * 8 * VPT;
@@ -143,17 +148,31 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
             // what sits in each stage, so that it can be stored out once the consumers are done with it
             uint16_t* held_out[STAGES][5];
             uint32_t held_bytes[STAGES];
+            uint32_t held_tensor[STAGES];      // for the replica copies of theta (multi-tensor plans only)
+            uint64_t held_elem[STAGES];
 #pragma unroll
-            for (int s = 0; s < STAGES; ++s) held_bytes[s] = 0;
+            for (int s = 0; s < STAGES; ++s) {
+                held_bytes[s] = 0;
+                held_tensor[s] = 0;
+                held_elem[s] = 0;
+            }
+            // theta of a finished tile also goes to every replica registered with the plan
+            auto store_replicas = [&](int s) {
+                if (FLAT) return;
+                for (int r = 0; r < p.num_replicas; ++r)
+                    pipe::bulk_store(replica_ptr(p, r, held_tensor[s], held_elem[s]), sm.data[s][0], held_bytes[s]);
+            };
 
             for (uint64_t c = blockIdx.x; c < p.num_chunks && alive; c += gridDim.x) {
                 TensorRec t;
                 uint64_t start;
+                uint32_t tensor_id = 0;
                 if (FLAT) {
                     t = p.flat;
                     start = c * p.chunk_elems;
                 } else {
                     const ChunkRec cr = p.chunks[c];
+                    tensor_id = cr.tensor;
                     t = p.tensors[cr.tensor];
                     start = static_cast<uint64_t>(cr.index) * p.chunk_elems;
                 }
@@ -168,6 +187,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                         if (held_bytes[s]) {
 #pragma unroll
                             for (int a = 0; a < NOUT; ++a) pipe::bulk_store(held_out[s][a], sm.data[s][a], held_bytes[s]);
+                            store_replicas(s);
                             pipe::bulk_commit();
                             pipe::bulk_wait_read_all();   // the stage may be overwritten once it has been read out
                         }
@@ -178,6 +198,8 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                         const uint16_t* g;
                         tile_pointers<STRATEGY>(t, start + off, held_out[s], g);
                         held_bytes[s] = kTile * 2;
+                        held_elem[s] = start + off;
+                        held_tensor[s] = tensor_id;
                         pipe::mbar_arrive_expect_tx(&sm.full[s], NIN * kTile * 2);
 #pragma unroll
                         for (int a = 0; a < NOUT; ++a) pipe::bulk_load(sm.data[s][a], held_out[s][a], kTile * 2, &sm.full[s]);
@@ -197,6 +219,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                 if (held_bytes[s]) {
 #pragma unroll
                     for (int a = 0; a < NOUT; ++a) pipe::bulk_store(held_out[s][a], sm.data[s][a], held_bytes[s]);
+                    store_replicas(s);
                     pipe::bulk_commit();
                 }
             }
@@ -215,11 +238,13 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
         for (uint64_t c = blockIdx.x; c < p.num_chunks && alive; c += gridDim.x) {
             TensorRec t;
             uint64_t start;
+            uint32_t tensor_id = 0;
             if (FLAT) {
                 t = p.flat;
                 start = c * p.chunk_elems;
             } else {
                 const ChunkRec cr = p.chunks[c];
+                tensor_id = cr.tensor;
                 t = p.tensors[cr.tensor];
                 start = static_cast<uint64_t>(cr.index) * p.chunk_elems;
             }
@@ -264,12 +289,21 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                         compute_vec<STRATEGY, EDQ, FAST, VARIANT>(v, k, 8, dot, sq, lost);
                         if (t.aligned) store_vec<STRATEGY>(v, t, base + 8ull * i);
                         else store_elems<STRATEGY>(v, t, base + 8ull * i, 8);
+                        if (!FLAT)
+                            for (int r = 0; r < p.num_replicas; ++r) {
+                                uint16_t* dst = replica_ptr(p, r, tensor_id, base + 8ull * i);
+                                if (t.aligned) st_stream(dst, v.th);
+                                else st_elems(dst, v.th, 8);
+                            }
                     }
                     if (rem && threadIdx.x == (nvec % CONSUMERS)) {
                         Vec v;
                         load_elems<STRATEGY>(v, t, base + 8ull * nvec, rem);
                         compute_vec<STRATEGY, EDQ, FAST, VARIANT>(v, k, rem, dot, sq, lost);
                         store_elems<STRATEGY>(v, t, base + 8ull * nvec, rem);
+                        if (!FLAT)
+                            for (int r = 0; r < p.num_replicas; ++r)
+                                st_elems(replica_ptr(p, r, tensor_id, base + 8ull * nvec), v.th, rem);
                     }
                 }
                 __syncwarp();

@@ -50,6 +50,30 @@ def partition(sizes: list[int], world: int, align: int = 8) -> list[list[tuple[i
     return out
 
 
+def slice_rows(rows, ranges):
+    """Rows of a rank's own plan: the (x_hi, x_lo, m, v_hi, v_lo, grad, n) tuples of `rows` cut to `ranges`.
+
+    `rows` are the full tensors (torch tensors or None); `ranges` is one rank's entry of `partition`.
+    The result feeds `binding.plan_create`; element `begin` of a tensor stays 16-byte aligned whenever
+    the tensor is, because `partition` cuts at multiples of 8 elements.
+    """
+    out = []
+    for i, b, e in ranges:
+        cut = tuple(None if t is None else t[b:e] for t in rows[i][:6])
+        out.append(cut + (e - b,))
+    return out
+
+
+def replica_rows(peer_x_hi, ranges):
+    """For `binding.plan_set_replicas`: this rank's slices inside each peer's full copy of theta.
+
+    `peer_x_hi[r][i]` is tensor i of peer r's parameter copy, mapped into this process (its own memory for
+    a single-GPU test; a peer-access or symmetric-memory mapping on several GPUs).  Returns one list per
+    peer, aligned with `slice_rows(rows, ranges)`.
+    """
+    return [[peer[i][b:e] for i, b, e in ranges] for peer in peer_x_hi]
+
+
 def allreduce_edq(sums, dist=None, group=None) -> dict:
     """Add {dot, sumsq, lost} over ranks in place (a 3-element float64 tensor) and form EDQ.
 

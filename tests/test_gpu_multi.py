@@ -159,3 +159,46 @@ def test_per_tensor_edq_matches_oracle_tensor_by_tensor(strategy, chunk):
         B.adamw_step_multi_per_tensor(plan, B.make_hyper(**hyp), 1, strategy, per, num, cws[:64])
     assert err.value.status == B.ERR_WORKSPACE
     B.plan_destroy(plan)
+
+
+@pytest.mark.parametrize("strategy", [0, 2])
+def test_theta_replicas_are_written_by_the_step_itself(strategy):
+    # sharded optimizer state needs theta everywhere: the step writes it to registered replicas (here two more
+    # buffers on this GPU; on several GPUs they would be peers' memory) - ragged, unaligned and empty tensors included
+    shapes = W.ragged_shapes() + [("big", 500_003)]
+    hyp = W.HYPERS
+    mis = lambda i: (0, 0, 1, 0, 3)[i % 5]
+    host, dev, grads, rows = _build(shapes, strategy, seed=9, misalign_of=mis)
+    plan = B.plan_create(rows)
+    reps = [[Guarded(np.full(n, 0x7FC1, np.uint16), mis(i)) for i, (_, n) in enumerate(shapes)] for _ in range(2)]
+    B.plan_set_replicas(plan, [[g.t if g.n else None for g in rep] for rep in reps])
+    e = EdqBuffers()
+    for t in (1, 2):
+        gbits = _set_grads(shapes, grads, 9, t)
+        B.adamw_step_multi(plan, e.hyper(hyp), t, strategy)
+        torch.cuda.synchronize()
+        want = _oracle_multi(host, gbits, t, strategy, hyp)
+        for i, (st, d) in enumerate(zip(host, dev)):
+            assert_same_bits(d["x_hi"].bits(), st["x_hi"], f"tensor {i} theta step {t}")
+            for r, rep in enumerate(reps):
+                assert_same_bits(rep[i].bits(), st["x_hi"], f"replica {r} tensor {i} step {t}")
+                assert rep[i].guards_intact()
+        edq_close(e.read(), want)
+    # replicas must not overlap the plan's arrays, and must sit like their tensor modulo 16 bytes
+    with pytest.raises(B.CollageError) as err:
+        B.plan_set_replicas(plan, [[d["m"].t if d["m"].n else None for d in dev]])
+    assert err.value.status == B.ERR_ALIAS
+    bad = [[g.t if g.n else None for g in reps[0]]]
+    big = len(shapes) - 1
+    bad[0][big] = reps[0][big].raw[reps[0][big].lo + 1:].view(torch.bfloat16)
+    with pytest.raises(B.CollageError) as err:
+        B.plan_set_replicas(plan, bad)
+    assert err.value.status == B.ERR_ARG
+    B.plan_set_replicas(plan, [])                      # detach
+    gbits = _set_grads(shapes, grads, 9, 3)
+    before = [rep[-1].bits() for rep in reps]
+    B.adamw_step_multi(plan, e.hyper(hyp), 3, strategy)
+    torch.cuda.synchronize()
+    assert all(np.array_equal(b, rep[-1].bits()) for b, rep in zip(before, reps))
+    assert B.pipeline_fault() == 0
+    B.plan_destroy(plan)

@@ -102,3 +102,25 @@ def test_two_ranks_reproduce_the_global_edq():
         assert got["edq"] == pytest.approx(want_edq, rel=1e-12)      # both ranks hold the same global value
         assert got["lost"] == tot["lost"]
     assert sum(c for _, _, c in results) == checksum                  # the slices together are the whole state
+
+
+def test_slices_of_all_ranks_tile_every_tensor_and_keep_alignment():
+    sizes = [4096, 9, 100_003, 0, 65_536]
+    rows = []
+    for n in sizes:
+        ts = [torch.arange(n, dtype=torch.int32).to(torch.bfloat16) for _ in range(6)]
+        rows.append(tuple(ts) + (n,))
+    world = 3
+    parts = sharding.partition(sizes, world)
+    covered = [torch.zeros(n, dtype=torch.int32) for n in sizes]
+    for rank in range(world):
+        mine = sharding.slice_rows(rows, parts[rank])
+        reps = sharding.replica_rows([[r[0] for r in rows]], parts[rank])
+        assert len(mine) == len(parts[rank]) == len(reps[0])
+        for (i, b, e), row, rep in zip(parts[rank], mine, reps[0]):
+            assert row[6] == e - b and all(t.numel() == e - b for t in row[:6])
+            assert row[0].data_ptr() == rows[i][0].data_ptr() + 2 * b          # a view, not a copy
+            assert (row[0].data_ptr() - rows[i][0].data_ptr()) % 16 == 0        # alignment carried over
+            assert rep.data_ptr() == row[0].data_ptr()
+            covered[i][b:e] += 1
+    assert all(bool((c == 1).all()) for c in covered)
