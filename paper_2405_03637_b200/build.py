@@ -20,6 +20,7 @@ NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "-fmad=false", "-ftz=false", "-prec-div=true", "-prec-sqrt=true",
     "-Xcompiler", "-fPIC", "-shared", "-cudart", "static",
+    "--split-compile", "0", "-t", "0",      # compile the many kernel instantiations on all host cores
 ]
 
 

@@ -108,7 +108,7 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
     uint32_t* dv = reinterpret_cast<uint32_t*>(&s.dv);
     const uint32_t* g = reinterpret_cast<const uint32_t*>(&s.g);
     EdqAcc acc = {0ull, 0ull, 0u};
-    if (STRATEGY == 4) {
+    if constexpr (STRATEGY == 4) {
         // float arithmetic in registers: lane by lane, then the same EDQ terms on the stored pairs
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -151,44 +151,44 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
             sq += static_cast<double>(edq_sq(acc));
             lost += acc.lost;
         }
-        return;
-    }
+    } else {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        ElemState e;
-        e.th = th[j];
-        e.dth = stores_x_lo(STRATEGY) ? dth[j] : 0u;   // delta-theta (B, C) or the Kahan compensation
-        e.m = m[j];
-        e.v = v[j];
-        e.dv = stores_v_lo(STRATEGY) ? dv[j] : 0u;
-        const bf2 th_old = e.th, dth_old = e.dth;
-        const PairUpdate up = adamw_pair<STRATEGY, FAST, VARIANT>(e, g[j], k);
-        th[j] = e.th;
-        m[j] = e.m;
-        v[j] = e.v;
-        if (stores_x_lo(STRATEGY)) dth[j] = e.dth;
-        if (stores_v_lo(STRATEGY)) dv[j] = e.dv;
-        if (EDQ) {
-            bf2 th_new = e.th, dth_new = e.dth, delta = up.delta, decay = up.decay;
-            if (valid < 8) {            // padded lanes hold zeros on input; keep them out of the sums
-                const int lanes = valid - 2 * j;
-                const uint32_t mask = lanes >= 2 ? 0xFFFFFFFFu : (lanes == 1 ? 0x0000FFFFu : 0u);
-                delta &= mask;
-                decay &= mask;
-                th_new &= mask;
-                dth_new &= mask;
+        for (int j = 0; j < 4; ++j) {
+            ElemState e;
+            e.th = th[j];
+            e.dth = stores_x_lo(STRATEGY) ? dth[j] : 0u;   // delta-theta (B, C) or the Kahan compensation
+            e.m = m[j];
+            e.v = v[j];
+            e.dv = stores_v_lo(STRATEGY) ? dv[j] : 0u;
+            const bf2 th_old = e.th, dth_old = e.dth;
+            const PairUpdate up = adamw_pair<STRATEGY, FAST, VARIANT>(e, g[j], k);
+            th[j] = e.th;
+            m[j] = e.m;
+            v[j] = e.v;
+            if (stores_x_lo(STRATEGY)) dth[j] = e.dth;
+            if (stores_v_lo(STRATEGY)) dv[j] = e.dv;
+            if (EDQ) {
+                bf2 th_new = e.th, dth_new = e.dth, delta = up.delta, decay = up.decay;
+                if (valid < 8) {            // padded lanes hold zeros on input; keep them out of the sums
+                    const int lanes = valid - 2 * j;
+                    const uint32_t mask = lanes >= 2 ? 0xFFFFFFFFu : (lanes == 1 ? 0x0000FFFFu : 0u);
+                    delta &= mask;
+                    decay &= mask;
+                    th_new &= mask;
+                    dth_new &= mask;
+                }
+                // intended update: line 12, plus the separate decay term when there is one
+                f32x2 d = widen2(delta);
+                if (VARIANT && (k.flags & 4u)) d = add_f32x2(d, widen2(decay));
+                // the stored parameter is the pair for options B and C, theta alone for A and Kahan
+                edq_pair_f<parameter_is_pair(STRATEGY)>(acc, th_old, dth_old, th_new, dth_new, d);
             }
-            // intended update: line 12, plus the separate decay term when there is one
-            f32x2 d = widen2(delta);
-            if (VARIANT && (k.flags & 4u)) d = add_f32x2(d, widen2(decay));
-            // the stored parameter is the pair for options B and C, theta alone for A and Kahan
-            edq_pair_f<parameter_is_pair(STRATEGY)>(acc, th_old, dth_old, th_new, dth_new, d);
         }
-    }
-    if (EDQ) {
-        dot += static_cast<double>(edq_dot(acc));
-        sq += static_cast<double>(edq_sq(acc));
-        lost += acc.lost;
+        if (EDQ) {
+            dot += static_cast<double>(edq_dot(acc));
+            sq += static_cast<double>(edq_sq(acc));
+            lost += acc.lost;
+        }
     }
 }
 

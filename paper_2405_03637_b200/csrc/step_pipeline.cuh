@@ -158,9 +158,10 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
             }
             // theta of a finished tile also goes to every replica registered with the plan
             auto store_replicas = [&](int s) {
-                if (FLAT) return;
-                for (int r = 0; r < p.num_replicas; ++r)
-                    pipe::bulk_store(replica_ptr(p, r, held_tensor[s], held_elem[s]), sm.data[s][0], held_bytes[s]);
+                if constexpr (!FLAT) {
+                    for (int r = 0; r < p.num_replicas; ++r)
+                        pipe::bulk_store(replica_ptr(p, r, held_tensor[s], held_elem[s]), sm.data[s][0], held_bytes[s]);
+                }
             };
 
             for (uint64_t c = blockIdx.x; c < p.num_chunks && alive; c += gridDim.x) {
