@@ -7,6 +7,7 @@
 // shared memory (cp.async.bulk + mbarrier, three stages), 512 consumers compute and write back, the
 // producer bulk-stores.  Traffic per parameter: D 28 B (reads g 2, m 4, v 4, w 4; writes theta 2,
 // m 4, v 4, w 4), D^-MW 22 B.
+#include "bulk_pipe.cuh"
 #include "host_common.cuh"
 #include "mcf_device.cuh"
 
@@ -18,59 +19,6 @@ void launch_edq_finalize(const EdqPartial* partials, int count, uint64_t n, coll
 // collage_pipeline_fault reports it together with the bfloat16 step's
 static __device__ unsigned int g_pipeline_fault32 = 0;
 
-namespace pipe32 {
-// the same bounded-wait helpers as the bfloat16 pipeline, kept local to this translation unit
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_addr(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// gives up after ~4e9 cycles (about two seconds) and records which wait failed
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int who) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 256; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > 4000000000LL) {
-            atomicCAS(&g_pipeline_fault32, 0u, who + 1u);
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_addr(smem_dst)),
-                 "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar))
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gmem_dst), "r"(smem_addr(smem_src)),
-                 "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-}  // namespace pipe32
 
 struct Fp32Scalars {
     float b1, c1, b2, c2, bc1, bc2, neg_a, lam, eps;
@@ -164,10 +112,10 @@ __global__ void __launch_bounds__(kCons32 + 32, 1) adamw_fp32_pipeline_kernel(co
     if (threadIdx.x == 0) {
 #pragma unroll
         for (int s = 0; s < kStages32; ++s) {
-            pipe32::mbar_init(&sm.full[s], 1);
-            pipe32::mbar_init(&sm.done[s], kWarps);
+            pipe::mbar_init(&sm.full[s], 1);
+            pipe::mbar_init(&sm.done[s], kWarps);
         }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        pipe::mbar_init_fence();
     }
     __syncthreads();
 
@@ -189,21 +137,21 @@ __global__ void __launch_bounds__(kCons32 + 32, 1) adamw_fp32_pipeline_kernel(co
             }
             auto store_out = [&](int s) {
                 const uint64_t off = held[s] * kTile32;
-                pipe32::bulk_store(p.theta + off, sm.stage[s].theta, kTile32 * 2);
-                pipe32::bulk_store(p.m + off, sm.stage[s].m, kTile32 * 4);
-                pipe32::bulk_store(p.v + off, sm.stage[s].v, kTile32 * 4);
-                if (MASTER) pipe32::bulk_store(p.master + off, sm.stage[s].w, kTile32 * 4);
-                pipe32::bulk_commit();
+                pipe::bulk_store(p.theta + off, sm.stage[s].theta, kTile32 * 2);
+                pipe::bulk_store(p.m + off, sm.stage[s].m, kTile32 * 4);
+                pipe::bulk_store(p.v + off, sm.stage[s].v, kTile32 * 4);
+                if (MASTER) pipe::bulk_store(p.master + off, sm.stage[s].w, kTile32 * 4);
+                pipe::bulk_commit();
             };
             for (uint64_t tile = blockIdx.x; tile < num_tiles && alive; tile += gridDim.x, ++it) {
                 const int s = it % kStages32;
                 const uint32_t use = it / kStages32;
                 if (use > 0) {
-                    alive = pipe32::mbar_wait(&sm.done[s], (use - 1) & 1u, 60u + s);
+                    alive = pipe::mbar_wait(&sm.done[s], (use - 1) & 1u, 60u + s, &g_pipeline_fault32);
                     if (!alive) break;
                     if (held_bulk[s]) {
                         store_out(s);
-                        pipe32::bulk_wait_read_all();
+                        pipe::bulk_wait_read_all();
                     }
                 }
                 const uint64_t off = tile * kTile32;
@@ -212,34 +160,34 @@ __global__ void __launch_bounds__(kCons32 + 32, 1) adamw_fp32_pipeline_kernel(co
                 held_bulk[s] = bulk;
                 if (bulk) {
                     const uint32_t bytes = kTile32 * (2 + 4 + 4 + (MASTER ? 4 : 2));
-                    pipe32::mbar_arrive_expect_tx(&sm.full[s], bytes);
-                    pipe32::bulk_load(sm.stage[s].g, p.grad + off, kTile32 * 2, &sm.full[s]);
-                    pipe32::bulk_load(sm.stage[s].m, p.m + off, kTile32 * 4, &sm.full[s]);
-                    pipe32::bulk_load(sm.stage[s].v, p.v + off, kTile32 * 4, &sm.full[s]);
-                    if (MASTER) pipe32::bulk_load(sm.stage[s].w, p.master + off, kTile32 * 4, &sm.full[s]);
-                    else pipe32::bulk_load(sm.stage[s].theta, p.theta + off, kTile32 * 2, &sm.full[s]);
+                    pipe::mbar_arrive_expect_tx(&sm.full[s], bytes);
+                    pipe::bulk_load(sm.stage[s].g, p.grad + off, kTile32 * 2, &sm.full[s]);
+                    pipe::bulk_load(sm.stage[s].m, p.m + off, kTile32 * 4, &sm.full[s]);
+                    pipe::bulk_load(sm.stage[s].v, p.v + off, kTile32 * 4, &sm.full[s]);
+                    if (MASTER) pipe::bulk_load(sm.stage[s].w, p.master + off, kTile32 * 4, &sm.full[s]);
+                    else pipe::bulk_load(sm.stage[s].theta, p.theta + off, kTile32 * 2, &sm.full[s]);
                 } else {
-                    pipe32::mbar_arrive(&sm.full[s]);
+                    pipe::mbar_arrive(&sm.full[s]);
                 }
             }
             const uint32_t tail = it < static_cast<uint32_t>(kStages32) ? it : kStages32;
             for (uint32_t j = it - tail; j < it && alive; ++j) {
                 const int s = j % kStages32;
-                alive = pipe32::mbar_wait(&sm.done[s], (j / kStages32) & 1u, 70u + s);
+                alive = pipe::mbar_wait(&sm.done[s], (j / kStages32) & 1u, 70u + s, &g_pipeline_fault32);
                 if (!alive) break;
                 if (held_bulk[s]) store_out(s);
             }
             if (!alive) {
                 for (int s = 0; s < kStages32; ++s)
-                    if (it > static_cast<uint32_t>(s)) pipe32::mbar_wait(&sm.full[s], ((it - 1 - s) / kStages32) & 1u, 80u + s);
+                    if (it > static_cast<uint32_t>(s)) pipe::mbar_wait(&sm.full[s], ((it - 1 - s) / kStages32) & 1u, 80u + s, &g_pipeline_fault32);
             }
-            pipe32::bulk_wait_all();
+            pipe::bulk_wait_all();
         }
     } else {
         const int lane = threadIdx.x & 31;
         for (uint64_t tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
             const int s = it % kStages32;
-            alive = __all_sync(0xFFFFFFFFu, pipe32::mbar_wait(&sm.full[s], (it / kStages32) & 1u, 90u + s));
+            alive = __all_sync(0xFFFFFFFFu, pipe::mbar_wait(&sm.full[s], (it / kStages32) & 1u, 90u + s, &g_pipeline_fault32));
             if (!alive) break;
             const uint64_t off = tile * kTile32;
             Fp32Acc acc = {0.0f, 0.0f, 0u};
@@ -270,7 +218,7 @@ __global__ void __launch_bounds__(kCons32 + 32, 1) adamw_fp32_pipeline_kernel(co
                     if (MASTER) *reinterpret_cast<float4*>(&st.w[e]) = w4;
                     *reinterpret_cast<uint2*>(&st.theta[e]) = make_uint2(tw[0], tw[1]);
                 }
-                pipe32::fence_async_smem();
+                pipe::fence_async_smem();
             } else {
                 // ragged last tile or unaligned arrays: element by element, straight from global memory
                 const uint64_t end = (p.n - off) < static_cast<uint64_t>(kTile32) ? p.n : off + kTile32;
@@ -290,7 +238,7 @@ __global__ void __launch_bounds__(kCons32 + 32, 1) adamw_fp32_pipeline_kernel(co
                 lost += acc.lost;
             }
             __syncwarp();
-            if (lane == 0) pipe32::mbar_arrive(&sm.done[s]);
+            if (lane == 0) pipe::mbar_arrive(&sm.done[s]);
         }
     }
 

@@ -14,67 +14,13 @@
 // tensor) flow through the same barriers but are processed straight from global memory.
 // Every wait is bounded: after ~2 s a thread records a fault in g_pipeline_fault and leaves.
 #pragma once
+#include "bulk_pipe.cuh"
 #include "mcf_device.cuh"
 
 namespace collage {
 
 __device__ unsigned int g_pipeline_fault = 0;   // 0 = none; else 1 + index of the wait that gave up
 
-namespace pipe {
-
-__device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_addr(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: gives up after ~4e9 cycles (about two seconds), records which wait failed.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int who) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (;;) {
-#pragma unroll 1
-        for (int i = 0; i < 256; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > 4000000000LL) {
-            atomicCAS(&g_pipeline_fault, 0u, who + 1u);
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_addr(smem_dst)),
-                 "l"(gmem_src), "r"(bytes), "r"(smem_addr(bar))
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gmem_dst), "r"(smem_addr(smem_src)),
-                 "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-}  // namespace pipe
 
 // Number of state arrays read / written per option
 template <int STRATEGY>
@@ -133,7 +79,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
         }
         pipe::mbar_init(&sm.red_full, kWarps);
         pipe::mbar_init(&sm.red_free, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        pipe::mbar_init_fence();
     }
     __syncthreads();
 
@@ -183,7 +129,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                     const int s = it % STAGES;
                     const uint32_t use = it / STAGES;
                     if (use > 0) {   // the stage still holds tile it - STAGES: wait for it, send it home
-                        alive = pipe::mbar_wait(&sm.done[s], (use - 1) & 1u, 10u + s);
+                        alive = pipe::mbar_wait(&sm.done[s], (use - 1) & 1u, 10u + s, &g_pipeline_fault);
                         if (!alive) break;
                         if (held_bytes[s]) {
 #pragma unroll
@@ -215,7 +161,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
             const uint32_t tail = it < static_cast<uint32_t>(STAGES) ? it : STAGES;
             for (uint32_t j = it - tail; j < it && alive; ++j) {
                 const int s = j % STAGES;
-                alive = pipe::mbar_wait(&sm.done[s], (j / STAGES) & 1u, 20u + s);
+                alive = pipe::mbar_wait(&sm.done[s], (j / STAGES) & 1u, 20u + s, &g_pipeline_fault);
                 if (!alive) break;
                 if (held_bytes[s]) {
 #pragma unroll
@@ -228,7 +174,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                 // a wait gave up: loads already issued still land in shared memory; let them finish
                 for (int s = 0; s < STAGES; ++s) {
                     const uint32_t armed = (it > static_cast<uint32_t>(s)) ? (it - 1 - s) / STAGES : 0;
-                    if (it > static_cast<uint32_t>(s)) pipe::mbar_wait(&sm.full[s], armed & 1u, 30u + s);
+                    if (it > static_cast<uint32_t>(s)) pipe::mbar_wait(&sm.full[s], armed & 1u, 30u + s, &g_pipeline_fault);
                 }
             }
             pipe::bulk_wait_all();
@@ -254,7 +200,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
             for (uint32_t off = 0; off < len; off += kTile, ++it) {
                 const int s = it % STAGES;
                 // a wait that gives up must take the whole warp with it (the lanes meet again in __syncwarp)
-                alive = __all_sync(0xFFFFFFFFu, pipe::mbar_wait(&sm.full[s], (it / STAGES) & 1u, 40u + s));
+                alive = __all_sync(0xFFFFFFFFu, pipe::mbar_wait(&sm.full[s], (it / STAGES) & 1u, 40u + s, &g_pipeline_fault));
                 if (!alive) break;
                 const uint32_t tl = (len - off) < static_cast<uint32_t>(kTile) ? (len - off) : kTile;
                 if (t.aligned && tl == static_cast<uint32_t>(kTile)) {
@@ -322,7 +268,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                     lost64 += __shfl_down_sync(0xFFFFFFFFu, lost64, o);
                 }
                 if (chunks_done > 0)
-                    alive = __all_sync(0xFFFFFFFFu, pipe::mbar_wait(&sm.red_free, (chunks_done - 1) & 1u, 50u));
+                    alive = __all_sync(0xFFFFFFFFu, pipe::mbar_wait(&sm.red_free, (chunks_done - 1) & 1u, 50u, &g_pipeline_fault));
                 if (alive) {
                     if (lane == 0) {
                         sm.red_dot[threadIdx.x >> 5] = dot;
@@ -331,7 +277,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                         pipe::mbar_arrive(&sm.red_full);
                     }
                     if (threadIdx.x == 0) {
-                        if (pipe::mbar_wait(&sm.red_full, chunks_done & 1u, 51u)) {
+                        if (pipe::mbar_wait(&sm.red_full, chunks_done & 1u, 51u, &g_pipeline_fault)) {
                             double d = 0.0, q = 0.0;
                             unsigned long long l = 0;
 #pragma unroll
