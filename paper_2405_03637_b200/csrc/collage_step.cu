@@ -97,8 +97,11 @@ struct Vec {
     uint4 th, dth, m, v, dv, g;
 };
 
-// The arithmetic of 8 parameters held in registers.  `valid` < 8 masks padded lanes out of EDQ.
-template <int STRATEGY, bool EDQ, bool FAST, bool VARIANT = false>
+// The arithmetic of 8 parameters held in registers, every operand answered in place (the rare
+// lanes by branches).  `valid` < 8 masks padded lanes out of EDQ.  FAST as in update_ratio, except
+// that a lane it cannot answer is NOT repeated here: callers that pass FAST = true use
+// compute_vec_fast below instead.
+template <int STRATEGY, bool EDQ, bool VARIANT = false>
 __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int valid, double& dot, double& sq,
                                             uint32_t& lost) {
     uint32_t* th = reinterpret_cast<uint32_t*>(&s.th);
@@ -146,12 +149,8 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
                 edq_pair_f<true>(acc, th_old, dth_old, th_new, dth_new, d);
             }
         }
-        if (EDQ) {
-            dot += static_cast<double>(edq_dot(acc));
-            sq += static_cast<double>(edq_sq(acc));
-            lost += acc.lost;
-        }
     } else {
+        uint32_t unused = 0u;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             ElemState e;
@@ -161,7 +160,7 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
             e.v = v[j];
             e.dv = stores_v_lo(STRATEGY) ? dv[j] : 0u;
             const bf2 th_old = e.th, dth_old = e.dth;
-            const PairUpdate up = adamw_pair<STRATEGY, FAST, VARIANT>(e, g[j], k);
+            const PairUpdate up = adamw_pair<STRATEGY, false, VARIANT>(e, g[j], k, unused);
             th[j] = e.th;
             m[j] = e.m;
             v[j] = e.v;
@@ -184,12 +183,99 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
                 edq_pair_f<parameter_is_pair(STRATEGY)>(acc, th_old, dth_old, th_new, dth_new, d);
             }
         }
+    }
+    if (EDQ) {
+        dot += static_cast<double>(edq_dot(acc));
+        sq += static_cast<double>(edq_sq(acc));
+        lost += acc.lost;
+    }
+}
+
+// The same for a full vector on the host-validated fast chain, without a branch: returns nonzero
+// when some lane holds a quotient or root that the fast chain cannot answer.  The caller then
+// discards `s` and `acc` and repeats the vector with compute_vec.
+template <int STRATEGY, bool EDQ, bool VARIANT = false>
+__device__ __forceinline__ uint32_t compute_vec_fast(Vec& s, const StepScalars& k, double& dot, double& sq, uint32_t& lost) {
+    static_assert(STRATEGY != 4, "the register variant has no fast chain");
+    uint32_t* th = reinterpret_cast<uint32_t*>(&s.th);
+    uint32_t* dth = reinterpret_cast<uint32_t*>(&s.dth);
+    uint32_t* m = reinterpret_cast<uint32_t*>(&s.m);
+    uint32_t* v = reinterpret_cast<uint32_t*>(&s.v);
+    uint32_t* dv = reinterpret_cast<uint32_t*>(&s.dv);
+    const uint32_t* g = reinterpret_cast<const uint32_t*>(&s.g);
+    EdqAcc acc = {0ull, 0ull, 0u};
+    uint32_t suspect = 0u;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        ElemState e;
+        e.th = th[j];
+        e.dth = stores_x_lo(STRATEGY) ? dth[j] : 0u;
+        e.m = m[j];
+        e.v = v[j];
+        e.dv = stores_v_lo(STRATEGY) ? dv[j] : 0u;
+        const bf2 th_old = e.th, dth_old = e.dth;
+        const PairUpdate up = adamw_pair<STRATEGY, true, VARIANT>(e, g[j], k, suspect);
+        th[j] = e.th;
+        m[j] = e.m;
+        v[j] = e.v;
+        if (stores_x_lo(STRATEGY)) dth[j] = e.dth;
+        if (stores_v_lo(STRATEGY)) dv[j] = e.dv;
         if (EDQ) {
-            dot += static_cast<double>(edq_dot(acc));
-            sq += static_cast<double>(edq_sq(acc));
-            lost += acc.lost;
+            f32x2 d = widen2(up.delta);
+            bf2 asked = up.delta;
+            if (VARIANT && (k.flags & 4u)) {
+                d = add_f32x2(d, widen2(up.decay));
+                asked = add2(up.delta, up.decay);       // zero exactly where the float sum is
+            }
+            edq_pair_packed<parameter_is_pair(STRATEGY)>(acc, th_old, dth_old, e.th, e.dth, d, asked);
         }
     }
+    if (EDQ && suspect == 0u) {
+        dot += static_cast<double>(edq_dot(acc));
+        sq += static_cast<double>(edq_sq(acc));
+        lost += edq_lost_packed(acc);
+    }
+    return suspect;
+}
+
+// One vector of a tile staged in shared memory: array a of the tile starts at tile + a * TILE, in
+// the order theta, m, v, [delta-theta], [delta-v], g.
+template <int STRATEGY, int TILE>
+__device__ __forceinline__ Vec tile_vector_load(const uint16_t* tile) {
+    Vec r;
+    int a = 0;
+    r.th = *reinterpret_cast<const uint4*>(tile + TILE * a++);
+    r.m = *reinterpret_cast<const uint4*>(tile + TILE * a++);
+    r.v = *reinterpret_cast<const uint4*>(tile + TILE * a++);
+    if (stores_x_lo(STRATEGY)) r.dth = *reinterpret_cast<const uint4*>(tile + TILE * a++);
+    if (stores_v_lo(STRATEGY)) r.dv = *reinterpret_cast<const uint4*>(tile + TILE * a++);
+    r.g = *reinterpret_cast<const uint4*>(tile + TILE * a);
+    return r;
+}
+template <int STRATEGY, int TILE>
+__device__ __forceinline__ void tile_vector_store(uint16_t* tile, const Vec& r) {
+    int a = 0;
+    *reinterpret_cast<uint4*>(tile + TILE * a++) = r.th;
+    *reinterpret_cast<uint4*>(tile + TILE * a++) = r.m;
+    *reinterpret_cast<uint4*>(tile + TILE * a++) = r.v;
+    if (stores_x_lo(STRATEGY)) *reinterpret_cast<uint4*>(tile + TILE * a++) = r.dth;
+    if (stores_v_lo(STRATEGY)) *reinterpret_cast<uint4*>(tile + TILE * a++) = r.dv;
+}
+
+// A vector that compute_vec_fast gave up on, repeated in place in the tile by the careful routes.
+// Out of line on purpose: it runs for a vanishing share of the vectors and must not weigh on the
+// register allocation of the loop that calls it.
+struct VecSums {
+    double dot, sq;
+    uint32_t lost;
+};
+template <int STRATEGY, bool EDQ, bool VARIANT, int TILE>
+__device__ __noinline__ VecSums careful_vector_in_tile(uint16_t* tile, const StepScalars& k) {
+    VecSums r = {0.0, 0.0, 0u};
+    Vec v = tile_vector_load<STRATEGY, TILE>(tile);
+    compute_vec<STRATEGY, EDQ, VARIANT>(v, k, 8, r.dot, r.sq, r.lost);
+    tile_vector_store<STRATEGY, TILE>(tile, v);
+    return r;
 }
 
 template <int STRATEGY>

@@ -224,6 +224,48 @@ __device__ __forceinline__ bf2 sqrt2_flushing(bf2 a) {
 #endif
 }
 
+// ---- deferred forms: no branch; a lane the fast route cannot answer sets bits in `suspect`, and
+// the caller recomputes the whole vector by the careful routes when any bit is set ---------------
+__device__ __forceinline__ uint32_t less_equal2(bf2 a, bf2 b) {
+    uint32_t d;
+    asm("set.le.u32.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// all-ones where the halves differ or either is NaN
+__device__ __forceinline__ uint32_t differs2(bf2 a, bf2 b) {
+    uint32_t d;
+    asm("set.neu.u32.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+__device__ __forceinline__ uint32_t equal2(bf2 a, bf2 b) {
+    uint32_t d;
+    asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// a (/) b under div2_normal_divisor's guarantee on b.  The rounded quotient is trusted unless its
+// magnitude is at most 2^-125 (the float product may then have been subnormal or tied) while the
+// numerator is not zero; a zero numerator gives the correctly signed zero (or NaN for a NaN
+// divisor) by the product alone, and a NaN product is a NaN quotient for every admitted divisor.
+__device__ __forceinline__ bf2 div2_normal_divisor_deferred(bf2 a, bf2 b, uint32_t& suspect) {
+#ifdef COLLAGE_IEEE_DIV_SQRT
+    return div2_ieee(a, b);
+#else
+    const bf2 q = pack_rn(__fmul_rn(hi_f32(a), rcp_ftz(hi_f32(b))), __fmul_rn(lo_f32(a), rcp_ftz(lo_f32(b))));
+    suspect |= less_equal2(q & 0x7FFF7FFFu, 0x01000100u) & ~equal2(a, 0u);   // 0x0100 = 2^-125
+    return q;
+#endif
+}
+// sqrt(a) under sqrt2_flushing's contract; a negative lane (NaN by IEEE, but -0 from the flushing
+// approximation when subnormal) marks the vector
+__device__ __forceinline__ bf2 sqrt2_flushing_deferred(bf2 a, uint32_t& suspect) {
+#ifdef COLLAGE_IEEE_DIV_SQRT
+    return sqrt2_ieee(a);
+#else
+    suspect |= less_than2(a, 0u);
+    return pack_rn(sqrt_ftz(hi_f32(a)), sqrt_ftz(lo_f32(a)));
+#endif
+}
+
 // --------------------------------------------------------- MCF algorithms ---
 
 struct bf2pair {
@@ -326,15 +368,17 @@ __host__ __device__ constexpr bool parameter_is_pair(int strategy) { return stra
 // denominator is NaN, Inf or >= eps, hence a valid operand of div2_normal_divisor, and (iii) with
 // epsilon outside the root a subnormal v-hat may be flushed by the root approximation: its root is
 // below 2^-63 < ulp(eps)/2 and is absorbed by the addition of eps either way.
+// With FAST the rare lanes are not answered here: they set bits in `suspect` (see the deferred
+// forms above) and the caller repeats the vector with FAST = false, which never touches `suspect`.
 template <bool FAST>
-__device__ __forceinline__ bf2 update_ratio(bf2 m, bf2 v, const StepScalars& k) {
+__device__ __forceinline__ bf2 update_ratio(bf2 m, bf2 v, const StepScalars& k, uint32_t& suspect) {
     bf2 mhat, vhat, den;
     if (FAST) {
         mhat = div2_by_scalar(m, k.rbc1);
         vhat = div2_by_scalar(v, k.rbc2);
-        if (k.flags & 1u) den = sqrt2_flushing(add2(vhat, k.eps));   // v-hat + eps >= eps: never subnormal
-        else den = add2(sqrt2_flushing(vhat), k.eps);
-        return div2_normal_divisor(mhat, den);
+        if (k.flags & 1u) den = sqrt2_flushing_deferred(add2(vhat, k.eps), suspect);   // v-hat + eps >= eps: never subnormal
+        else den = add2(sqrt2_flushing_deferred(vhat, suspect), k.eps);
+        return div2_normal_divisor_deferred(mhat, den, suspect);
     }
     mhat = div2_scalar(m, k.bc1, k.rbc1);
     vhat = div2_scalar(v, k.bc2, k.rbc2);
@@ -354,7 +398,7 @@ struct PairUpdate {
 // VARIANT kernels honour flags bit 1 (the parameter Grow uses TwoSum) and bit 2 (decay by its own
 // addition); the others are compiled without either, so the common path carries no test for them.
 template <int STRATEGY, bool FAST, bool VARIANT>
-__device__ __forceinline__ PairUpdate adamw_pair(ElemState& s, bf2 g, const StepScalars& k) {
+__device__ __forceinline__ PairUpdate adamw_pair(ElemState& s, bf2 g, const StepScalars& k, uint32_t& suspect) {
     // line 8
     s.m = add2(mul2(k.b1, s.m), mul2(k.c1, g));
     // line 9
@@ -368,7 +412,7 @@ __device__ __forceinline__ PairUpdate adamw_pair(ElemState& s, bf2 g, const Step
         s.v = add2(mul2(k.b2, s.v), tv);
     }
     // lines 10-12
-    const bf2 r = update_ratio<FAST>(s.m, s.v, k);
+    const bf2 r = update_ratio<FAST>(s.m, s.v, k, suspect);
     const bf2 w = mul2(k.lam, s.th);
     const bool split_decay = VARIANT && (k.flags & 4u) != 0;
     PairUpdate up;
@@ -421,6 +465,25 @@ __device__ __forceinline__ void edq_pair_f(EdqAcc& acc, bf2 th_old, bf2 dth_old,
     acc.lost += (lo_of(d) != 0.0f && same0) ? 1u : 0u;
     acc.lost += (hi_of(d) != 0.0f && same1) ? 1u : 0u;
 }
+// The same with the comparisons of Definition 3.2 done on the packed bfloat16 values (widening is
+// exact, so they decide as the float comparisons do: zeros of either sign are equal, NaN equals
+// nothing and differs from zero).  `asked` is the intended update as a bfloat16 pair, zero where
+// `d` is.  acc.lost collects the two halves as packed 16-bit counts: see edq_lost_packed.
+template <bool HAS_LO>
+__device__ __forceinline__ void edq_pair_packed(EdqAcc& acc, bf2 th_old, bf2 dth_old, bf2 th_new, bf2 dth_new, f32x2 d,
+                                                bf2 asked) {
+    f32x2 e = sub_f32x2(widen2(th_new), widen2(th_old));
+    uint32_t unchanged = equal2(th_new, th_old);
+    if (HAS_LO) {
+        e = add_f32x2(e, sub_f32x2(widen2(dth_new), widen2(dth_old)));
+        unchanged &= equal2(dth_new, dth_old);
+    }
+    acc.dot = fma_f32x2(d, e, acc.dot);
+    acc.sq = fma_f32x2(d, d, acc.sq);
+    acc.lost += unchanged & differs2(asked, 0u) & 0x00010001u;
+}
+// the count held in packed form by edq_pair_packed (at most 65535 pairs between two calls)
+__device__ __forceinline__ uint32_t edq_lost_packed(const EdqAcc& a) { return (a.lost & 0xFFFFu) + (a.lost >> 16); }
 template <bool HAS_LO>
 __device__ __forceinline__ void edq_pair(EdqAcc& acc, bf2 th_old, bf2 dth_old, bf2 th_new, bf2 dth_new, bf2 delta) {
     edq_pair_f<HAS_LO>(acc, th_old, dth_old, th_new, dth_new, widen2(delta));

@@ -206,22 +206,25 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                 if (t.aligned && tl == static_cast<uint32_t>(kTile)) {
 #pragma unroll
                     for (int j = 0; j < VPT; ++j) {
-                        Vec v;
                         const int e = (j * CONSUMERS + threadIdx.x) * 8;
-                        int a = 0;
-                        v.th = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
-                        v.m = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
-                        v.v = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
-                        if (stores_x_lo(STRATEGY)) v.dth = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
-                        if (stores_v_lo(STRATEGY)) v.dv = *reinterpret_cast<const uint4*>(&sm.data[s][a++][e]);
-                        v.g = *reinterpret_cast<const uint4*>(&sm.data[s][a][e]);
-                        compute_vec<STRATEGY, EDQ, FAST, VARIANT>(v, k, 8, dot, sq, lost);
-                        a = 0;
-                        *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.th;
-                        *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.m;
-                        *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.v;
-                        if (stores_x_lo(STRATEGY)) *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.dth;
-                        if (stores_v_lo(STRATEGY)) *reinterpret_cast<uint4*>(&sm.data[s][a++][e]) = v.dv;
+                        if constexpr (FAST && STRATEGY != 4) {
+                            Vec v = tile_vector_load<STRATEGY, kTile>(&sm.data[s][0][e]);
+                            if (compute_vec_fast<STRATEGY, EDQ, VARIANT>(v, k, dot, sq, lost) == 0u) {
+                                tile_vector_store<STRATEGY, kTile>(&sm.data[s][0][e], v);
+                            } else {
+                                // rare: the tile still holds the inputs; repeat the vector out of line
+                                const VecSums r = careful_vector_in_tile<STRATEGY, EDQ, VARIANT, kTile>(&sm.data[s][0][e], k);
+                                if (EDQ) {
+                                    dot += r.dot;
+                                    sq += r.sq;
+                                    lost += r.lost;
+                                }
+                            }
+                        } else {
+                            Vec v = tile_vector_load<STRATEGY, kTile>(&sm.data[s][0][e]);
+                            compute_vec<STRATEGY, EDQ, VARIANT>(v, k, 8, dot, sq, lost);
+                            tile_vector_store<STRATEGY, kTile>(&sm.data[s][0][e], v);
+                        }
                     }
                     pipe::fence_async_smem();      // shared-memory writes must be visible to the bulk store
                 } else {
@@ -233,7 +236,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                         Vec v;
                         if (t.aligned) load_vec<STRATEGY>(v, t, base + 8ull * i);
                         else load_elems<STRATEGY>(v, t, base + 8ull * i, 8);
-                        compute_vec<STRATEGY, EDQ, FAST, VARIANT>(v, k, 8, dot, sq, lost);
+                        compute_vec<STRATEGY, EDQ, VARIANT>(v, k, 8, dot, sq, lost);
                         if (t.aligned) store_vec<STRATEGY>(v, t, base + 8ull * i);
                         else store_elems<STRATEGY>(v, t, base + 8ull * i, 8);
                         if (!FLAT)
@@ -246,7 +249,7 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
                     if (rem && threadIdx.x == (nvec % CONSUMERS)) {
                         Vec v;
                         load_elems<STRATEGY>(v, t, base + 8ull * nvec, rem);
-                        compute_vec<STRATEGY, EDQ, FAST, VARIANT>(v, k, rem, dot, sq, lost);
+                        compute_vec<STRATEGY, EDQ, VARIANT>(v, k, rem, dot, sq, lost);
                         store_elems<STRATEGY>(v, t, base + 8ull * nvec, rem);
                         if (!FLAT)
                             for (int r = 0; r < p.num_replicas; ++r)

@@ -280,3 +280,44 @@ def test_negative_second_moment_gives_nan_not_a_flushed_zero():
         torch.cuda.synchronize()
         oracle_step(st, g, 5, strategy, hyp)
         _compare(dev, st, f"negative v, strategy {strategy}")
+
+
+@pytest.mark.parametrize("strategy", [0, 1, 2])
+def test_sparse_rare_lanes_between_ordinary_ones_keep_state_edq_and_lost_exact(strategy):
+    # Ordinary training state with about one lane in a hundred that the lean chain cannot answer by itself
+    # (subnormal or zero first moments, huge or subnormal second moments: tiny and tied quotients), and as many
+    # parameters whose update is lost even as a pair (theta = 2^31 with delta-theta = +-2^20, zeros of either
+    # sign beside them).  Vectors with and without such a lane alternate inside every tile; several tiles and
+    # a ragged tail.  State bit for bit, EDQ sums within tolerance, the lost count exactly.
+    n, hyp = 300_007, dict(W.HYPERS, weight_decay=0.0)
+    rng = np.random.default_rng(1234 + strategy)
+    st = oracle_state(W.bits(W.flat_weights(n, 61)), strategy)
+    dev = _device_state(st)
+    e = EdqBuffers()
+
+    def step(t):
+        g = W.bits(W.flat_grads(n, 61, t))
+        g[rng.random(n) < 0.01] = 0
+        G = Guarded(g)
+        B.adamw_step(_t(dev["x_hi"]), _t(dev["x_lo"]), _t(dev["m"]), _t(dev["v_hi"]), _t(dev["v_lo"]), G.t, n,
+                     e.hyper(hyp), t, strategy)
+        torch.cuda.synchronize()
+        want = oracle_step(st, g, t, strategy, hyp)
+        edq_close(e.read(), want)
+        _compare(dev, st, f"sparse rare lanes, strategy {strategy}, step {t}")
+        return want
+
+    step(1)
+    # poke the rare lanes into the (identical) host and device copies
+    where = lambda p: np.flatnonzero(rng.random(n) < p)
+    i = where(0.01)
+    st["m"][i] = rng.choice(np.array([0x0000, 0x8000, 0x0001, 0x8003, 0x0080], np.uint16), i.size)
+    i = where(0.01)
+    st["v_hi"][i] = rng.choice(np.array([0x7F00, 0x7F7F, 0x0001, 0x007F, 0x0000], np.uint16), i.size)
+    i = where(0.01)
+    st["x_hi"][i] = rng.choice(np.array([0x4F00, 0xCF00], np.uint16), i.size)
+    if strategy >= 1:
+        st["x_lo"][i] = rng.choice(np.array([0x4980, 0xC980, 0x0000, 0x8000], np.uint16), i.size)
+    dev = _device_state(st)
+    lost = [step(t)["lost"] for t in (2, 3, 4)]
+    assert min(lost) > 0        # the poked parameters do lose updates, so the exact count is exercised
