@@ -16,20 +16,38 @@
 // of 80 launches): 512 consumer threads + one producer warp, one block per SM, three stages of
 // 4096-element tiles reached 6.47 TB/s; an earlier register-staged kernel (16-byte loads into
 // registers, 6 blocks of 128 threads per SM) 6.07 TB/s; smaller tiles, more stages or two blocks
-// per SM were slower.
+// per SM were slower; 8192-element tiles in two stages (the same bytes in flight) measured the same
+// within the 1 % run-to-run noise.
+// Six staged arrays (option C, the register variant):
 #ifndef COLLAGE_PIPE_CONSUMERS
 #define COLLAGE_PIPE_CONSUMERS 512
-#endif
-// Option A moves the fewest bytes per parameter, so its arithmetic weighs more: 768 consumers
-// (6144-element tiles) measured 6.67 TB/s against 5.96 TB/s with 512.
-#ifndef COLLAGE_PIPE_CONSUMERS_A
-#define COLLAGE_PIPE_CONSUMERS_A 768
 #endif
 #ifndef COLLAGE_PIPE_VPT
 #define COLLAGE_PIPE_VPT 1
 #endif
 #ifndef COLLAGE_PIPE_STAGES
 #define COLLAGE_PIPE_STAGES 3
+#endif
+// five staged arrays (option B, BF16-Kahan):
+#ifndef COLLAGE_PIPE_CONSUMERS_B
+#define COLLAGE_PIPE_CONSUMERS_B COLLAGE_PIPE_CONSUMERS
+#endif
+#ifndef COLLAGE_PIPE_VPT_B
+#define COLLAGE_PIPE_VPT_B COLLAGE_PIPE_VPT
+#endif
+#ifndef COLLAGE_PIPE_STAGES_B
+#define COLLAGE_PIPE_STAGES_B COLLAGE_PIPE_STAGES
+#endif
+// Option A moves the fewest bytes per parameter, so its arithmetic weighs more: 768 consumers
+// (6144-element tiles) measured 6.67 TB/s against 5.96 TB/s with 512.
+#ifndef COLLAGE_PIPE_CONSUMERS_A
+#define COLLAGE_PIPE_CONSUMERS_A 768
+#endif
+#ifndef COLLAGE_PIPE_VPT_A
+#define COLLAGE_PIPE_VPT_A COLLAGE_PIPE_VPT
+#endif
+#ifndef COLLAGE_PIPE_STAGES_A
+#define COLLAGE_PIPE_STAGES_A COLLAGE_PIPE_STAGES
 #endif
 #ifndef COLLAGE_PIPE_MINBLOCKS
 #define COLLAGE_PIPE_MINBLOCKS 1
@@ -38,9 +56,19 @@
 namespace collage {
 
 constexpr uint32_t kDefaultChunk = 24576;   // a whole number of tiles for every precision option (6 x 4096, 4 x 6144)
-// elements per tile of the pipeline kernel for a precision option
+// consumer threads, vectors per thread and tile, and stages of the pipeline kernel for a precision option
+struct PipeGeometry {
+    int consumers, vpt, stages;
+};
+constexpr PipeGeometry pipe_geometry(int strategy) {
+    return strategy == 0 ? PipeGeometry{COLLAGE_PIPE_CONSUMERS_A, COLLAGE_PIPE_VPT_A, COLLAGE_PIPE_STAGES_A}
+           : (strategy == 1 || strategy == 3)
+               ? PipeGeometry{COLLAGE_PIPE_CONSUMERS_B, COLLAGE_PIPE_VPT_B, COLLAGE_PIPE_STAGES_B}
+               : PipeGeometry{COLLAGE_PIPE_CONSUMERS, COLLAGE_PIPE_VPT, COLLAGE_PIPE_STAGES};
+}
+// elements per tile
 constexpr uint32_t pipe_tile(int strategy) {
-    return (strategy == 0 ? COLLAGE_PIPE_CONSUMERS_A : COLLAGE_PIPE_CONSUMERS) * 8u * COLLAGE_PIPE_VPT;
+    return static_cast<uint32_t>(pipe_geometry(strategy).consumers) * 8u * static_cast<uint32_t>(pipe_geometry(strategy).vpt);
 }
 
 struct TensorRec {
@@ -468,8 +496,8 @@ static collage_status_t make_scalars(const collage_hyper_t* hyper, uint64_t step
 
 template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, bool PER_CHUNK = false, bool VARIANT = false>
 static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t stream, int* grid_out) {
-    constexpr int CONSUMERS = STRATEGY == 0 ? COLLAGE_PIPE_CONSUMERS_A : COLLAGE_PIPE_CONSUMERS;
-    constexpr int VPT = COLLAGE_PIPE_VPT, STAGES = COLLAGE_PIPE_STAGES;
+    constexpr int CONSUMERS = pipe_geometry(STRATEGY).consumers;
+    constexpr int VPT = pipe_geometry(STRATEGY).vpt, STAGES = pipe_geometry(STRATEGY).stages;
     auto kernel = adamw_step_pipeline_kernel<STRATEGY, EDQ, FLAT, FAST, CONSUMERS, VPT, STAGES, PER_CHUNK, VARIANT>;
     constexpr size_t smem = sizeof(PipeSmem<CONSUMERS, VPT, STAGES, STRATEGY>) + 128;
     constexpr int threads = CONSUMERS + 32;
