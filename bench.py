@@ -28,9 +28,9 @@ BYTES_PER_PARAM = {0: 14, 1: 18, 2: 22}      # algorithmic HBM bytes per paramet
 STRATEGY = 2                                  # Collage-plus
 WORKLOAD = "llama7b_shaped_291_tensors_collage_plus_with_edq"
 # DRAM bytes per parameter of the step kernel from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum = 3.146 GB + 2.565 GB on the 262,148,096-parameter case, summary under
+# dram__bytes_write.sum = 3.146 GB + 2.567 GB on the 262,148,096-parameter case, summary under
 # profiles/); every byte is touched once, so traffic scales with the parameter count.
-NCU_TRAFFIC_BYTES_PER_PARAM = (3.146196e9 + 2.565302e9) / 262_148_096
+NCU_TRAFFIC_BYTES_PER_PARAM = (3.146235e9 + 2.567421e9) / 262_148_096
 
 
 def measured_hbm_peak():
