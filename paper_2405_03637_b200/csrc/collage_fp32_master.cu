@@ -37,24 +37,48 @@ struct Fp32Params {
     EdqPartial* partials;
 };
 
-constexpr int kCons32 = 512;              // consumer threads
-constexpr int kQuads32 = 2;               // groups of 4 consecutive elements per thread and tile
-constexpr int kTile32 = kCons32 * 4 * kQuads32;   // 4096 elements
-constexpr int kStages32 = 3;
-
-struct Fp32Stage {
-    alignas(128) float m[kTile32];
-    alignas(128) float v[kTile32];
-    alignas(128) float w[kTile32];
-    alignas(128) uint16_t theta[kTile32];
-    alignas(128) uint16_t g[kTile32];
+// Geometry of the pipeline (one block per SM, a producer warp beside the consumers).  The version
+// without master weights moves 22 B per parameter for the same IEEE divisions and root as the
+// 28 B one, so its arithmetic weighs more and it wants more consumer threads: measured on a flat
+// 2^30 tensor, 512 / 768 / 960 consumers gave 5.2 / 5.7 / 5.9 TB/s without master weights and
+// 6.3 / 6.4 / 6.3 TB/s with them.
+#ifndef COLLAGE_FP32_CONSUMERS
+#define COLLAGE_FP32_CONSUMERS 768
+#endif
+#ifndef COLLAGE_FP32_CONSUMERS_NO_MASTER
+#define COLLAGE_FP32_CONSUMERS_NO_MASTER 960
+#endif
+#ifndef COLLAGE_FP32_QUADS
+#define COLLAGE_FP32_QUADS 1
+#endif
+#ifndef COLLAGE_FP32_STAGES
+#define COLLAGE_FP32_STAGES 3
+#endif
+template <bool MASTER>
+struct Fp32Geometry {
+    static constexpr int kCons = MASTER ? COLLAGE_FP32_CONSUMERS : COLLAGE_FP32_CONSUMERS_NO_MASTER;   // consumer threads
+    static constexpr int kQuads = COLLAGE_FP32_QUADS;      // groups of 4 consecutive elements per thread and tile
+    static constexpr int kTile = kCons * 4 * kQuads;       // elements per tile
+    static constexpr int kStages = COLLAGE_FP32_STAGES;
 };
+
+template <bool MASTER>
+struct Fp32Stage {
+    static constexpr int kTile = Fp32Geometry<MASTER>::kTile;
+    alignas(128) float m[kTile];
+    alignas(128) float v[kTile];
+    alignas(128) float w[MASTER ? kTile : 32];
+    alignas(128) uint16_t theta[kTile];
+    alignas(128) uint16_t g[kTile];
+};
+template <bool MASTER>
 struct Fp32Smem {
-    Fp32Stage stage[kStages32];
-    alignas(8) uint64_t full[kStages32];
-    alignas(8) uint64_t done[kStages32];
-    double red_dot[kCons32 / 32], red_sq[kCons32 / 32];
-    unsigned long long red_lost[kCons32 / 32];
+    static constexpr int kStages = Fp32Geometry<MASTER>::kStages, kCons = Fp32Geometry<MASTER>::kCons;
+    Fp32Stage<MASTER> stage[kStages];
+    alignas(8) uint64_t full[kStages];
+    alignas(8) uint64_t done[kStages];
+    double red_dot[kCons / 32], red_sq[kCons / 32];
+    unsigned long long red_lost[kCons / 32];
 };
 
 // One parameter: Algorithm 2 lines 8-13 in float.  Returns the update; w is the stored float
@@ -104,9 +128,11 @@ __device__ __forceinline__ void fp32_element(float& m, float& v, float& w, uint1
 }
 
 template <bool MASTER, bool EDQ>
-__global__ void __launch_bounds__(kCons32 + 32, 1) adamw_fp32_pipeline_kernel(const __grid_constant__ Fp32Params p) {
+__global__ void __launch_bounds__(Fp32Geometry<MASTER>::kCons + 32, 1) adamw_fp32_pipeline_kernel(const __grid_constant__ Fp32Params p) {
+    constexpr int kCons32 = Fp32Geometry<MASTER>::kCons, kQuads32 = Fp32Geometry<MASTER>::kQuads;
+    constexpr int kTile32 = Fp32Geometry<MASTER>::kTile, kStages32 = Fp32Geometry<MASTER>::kStages;
     extern __shared__ unsigned char smem_raw[];
-    Fp32Smem& sm = *reinterpret_cast<Fp32Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
+    Fp32Smem<MASTER>& sm = *reinterpret_cast<Fp32Smem<MASTER>*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
     constexpr int kWarps = kCons32 / 32;
     const bool is_producer = threadIdx.x >= kCons32;
     if (threadIdx.x == 0) {
@@ -192,7 +218,7 @@ __global__ void __launch_bounds__(kCons32 + 32, 1) adamw_fp32_pipeline_kernel(co
             const uint64_t off = tile * kTile32;
             Fp32Acc acc = {0.0f, 0.0f, 0u};
             if (p.aligned && (p.n - off) >= static_cast<uint64_t>(kTile32)) {
-                Fp32Stage& st = sm.stage[s];
+                Fp32Stage<MASTER>& st = sm.stage[s];
 #pragma unroll
                 for (int q = 0; q < kQuads32; ++q) {
                     const int e = (q * kCons32 + threadIdx.x) * 4;
@@ -275,7 +301,8 @@ __global__ void __launch_bounds__(kCons32 + 32, 1) adamw_fp32_pipeline_kernel(co
 template <bool MASTER, bool EDQ>
 static cudaError_t launch_fp32(const Fp32Params& p, int sm_count, cudaStream_t stream, int* grid_out) {
     auto kernel = adamw_fp32_pipeline_kernel<MASTER, EDQ>;
-    constexpr size_t smem = sizeof(Fp32Smem) + 128;
+    constexpr size_t smem = sizeof(Fp32Smem<MASTER>) + 128;
+    constexpr int kTile32 = Fp32Geometry<MASTER>::kTile, kCons32 = Fp32Geometry<MASTER>::kCons;
     static bool ready[64] = {};
     int device = 0;
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return cudaErrorInvalidDevice;
