@@ -319,14 +319,14 @@ def run_size_sweep(args):
 
 
 def run_strategy_sweep(args):
-    """All precision options, the comparators and the step variants on one flat 2^30-parameter tensor."""
+    """All precision options, the comparators and the step variants on one flat tensor (2^30 parameters by default)."""
     import torch
     from paper_2405_03637_b200 import binding as B
     from paper_2405_03637_b200 import workloads as W
     device = torch.device("cuda", 0)
     torch.cuda.set_device(device)
     peak, _ = measured_hbm_peak()
-    n = 1 << 30
+    n = 1 << args.sweep_log2n
     x = W.flat_weights(n, 0, device)
     z = lambda: torch.zeros_like(x)
     xl, m, v, vl, g = z(), z(), z(), z(), W.flat_grads(n, 0, 1, device)
@@ -341,7 +341,7 @@ def run_strategy_sweep(args):
         for t in range(1, 4):
             call(t)
         torch.cuda.synchronize()
-        iters = 40
+        iters = args.sweep_iters
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
         ev[0].record(stream)
         for i in range(iters):
@@ -436,6 +436,8 @@ def main():
     ap.add_argument("--per-tensor", action="store_true", help="time the per-tensor EDQ variant of the step")
     ap.add_argument("--strategy-sweep", action="store_true", help="time every option, comparator and variant on a flat tensor")
     ap.add_argument("--size-sweep", action="store_true", help="flat-tensor size sweep instead of the benchmark")
+    ap.add_argument("--sweep-log2n", type=int, default=30, help="--strategy-sweep: log2 of the flat tensor's length")
+    ap.add_argument("--sweep-iters", type=int, default=40, help="--strategy-sweep: timed steps per case")
     args = ap.parse_args()
     if args.size_sweep:
         run_size_sweep(args)
