@@ -228,3 +228,40 @@ def test_effective_descent_quality_orders_the_precision_strategies():
     assert mean["A"] < 0.95 * mean["B"]                              # plain bfloat16 loses a visible share
     assert quality["Kahan"][0] == quality["A"][0]                    # first step: no compensation yet
     assert mean["A"] < mean["Kahan"] <= 1.05                         # later steps deliver what earlier ones lost
+
+
+@pytest.mark.parametrize("api", ["flat", "multi"])
+def test_one_tensor_longer_than_2_to_32_elements(api):
+    # index arithmetic past 32 bits: a single Collage-plus tensor of 2^32 + 20,483 parameters (51.5 GB of
+    # state), through the flat entry point and as a one-tensor plan; windows at the start, around 2^32 and
+    # at the ragged end bit for bit, the element count and the sign of the sums from the EDQ record
+    dev = torch.device("cuda")
+    n = (1 << 32) + 20_483
+    x = W.normal_bf16(n, 0.02, 9001, dev)
+    g = W.normal_bf16(n, 1e-3, 9002, dev)
+    xl, m, v, vl = (torch.zeros_like(x) for _ in range(4))
+    arrs = (x, xl, m, v, vl)
+    rng = np.random.default_rng(5)
+    wins = _windows(n, rng, 4096, 8) + [((1 << 32) - 2048, (1 << 32) + 2048), (n - 20_483 - 64, n - 20_483 + 64)]
+    st = {k: _gather(a, wins) for a, k in zip(arrs, KEYS)}
+    gs = _gather(g, wins)
+    e = EdqBuffers()
+    plan = B.plan_create([(x, xl, m, v, vl, g, n)]) if api == "multi" else None
+    for t in (1, 2):
+        if api == "multi":
+            B.adamw_step_multi(plan, e.hyper(W.HYPERS), t, B.PLUS)
+        else:
+            B.adamw_step(x, xl, m, v, vl, g, n, e.hyper(W.HYPERS), t, B.PLUS)
+        torch.cuda.synchronize()
+        oracle_step(st, gs, t, 2, W.HYPERS)
+        for a, k in zip(arrs, KEYS):
+            assert_same_bits(_gather(a, wins), st[k], f"{api} step {t} {k}")
+        got = e.read()
+        assert got["n"] == n and got["sumsq"] > 0 and got["edq"] > 0
+    # every parameter moved: none of the 2^32 + 20,483 was skipped (theta changes in its pair with probability ~1)
+    assert int((xl == 0).sum().item()) < n // 8
+    assert B.pipeline_fault() == 0
+    if plan is not None:
+        B.plan_destroy(plan)
+    del x, g, xl, m, v, vl, arrs
+    torch.cuda.empty_cache()

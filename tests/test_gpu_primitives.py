@@ -180,6 +180,33 @@ def test_standalone_edq_matches_oracle():
         assert got["lost"] == want["lost"] and got["n"] == n
 
 
+def test_standalone_edq_past_2_to_32_elements_is_the_sum_of_its_pieces():
+    # index arithmetic past 32 bits: the sums over 2^32 + 4,099 parameters equal those of two pieces taken by
+    # the same entry point (each piece below 2^32; small n is compared with the oracle above)
+    from paper_2405_03637_b200 import workloads as W
+    n = (1 << 32) + 4_099
+    old = W.normal_bf16(n, 0.02, 811, "cuda")
+    delta = W.normal_bf16(n, 1e-4, 812, "cuda")
+    new = old + delta
+    new[5::11] = old[5::11]                                          # lost updates on both sides of 2^32
+    out = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    ws = torch.empty(B.workspace_bytes(), dtype=torch.uint8, device="cuda")
+
+    def run(lo, hi):
+        B.edq(old[lo:hi], None, new[lo:hi], None, delta[lo:hi], hi - lo, out, ws)
+        torch.cuda.synchronize()
+        return B.read_edq(out)
+
+    whole, cut = run(0, n), (1 << 31) + 8
+    a, b = run(0, cut), run(cut, n)
+    assert whole["n"] == n and a["n"] + b["n"] == n
+    assert whole["lost"] == a["lost"] + b["lost"] and whole["lost"] >= n // 11
+    for k in ("dot", "sumsq"):
+        assert abs(whole[k] - (a[k] + b[k])) <= 1e-9 * abs(whole[k])
+    del old, new, delta
+    torch.cuda.empty_cache()
+
+
 def test_selftest_every_operand_pair():
     # all 2^32 operand pairs on the device: native packed ops and the reciprocal/root shortcuts vs IEEE references
     assert B.selftest() == dict(add=0, sub=0, mul=0, div=0, sqrt=0, scalar_div=0)
