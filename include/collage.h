@@ -300,7 +300,10 @@ collage_status_t collage_pipeline_fault(uint32_t* out_host);
  * patterns (2^32 pairs; 2^16 values for the root), the realisation used in the kernels with a
  * reference built from IEEE float/double arithmetic and one conversion to bfloat16:
  *   out_host[0] add  [1] sub  [2] mul            native packed bfloat16 instructions
- *   out_host[3] div  [4] sqrt                    reciprocal / root approximations vs div.rn, sqrt.rn
+ *   out_host[3] div  [4] sqrt                    reciprocal / root approximations vs div.rn, sqrt.rn,
+ *                                                both in the form that answers every operand and in the
+ *                                                branch-free form of the step kernel (whose unflagged
+ *                                                lanes must be right on all operands it admits)
  *   out_host[5] division by a scalar through a host-rounded reciprocal (divisors in (0, 1])
  * Each entry is the number of results that differ (NaNs compared as a class); all must be 0.
  * HOST output; allocates a few bytes, synchronises `stream`; takes about a second.

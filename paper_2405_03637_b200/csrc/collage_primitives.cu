@@ -265,6 +265,19 @@ __global__ void __launch_bounds__(256) selftest_kernel(unsigned long long* count
         c_sub += mismatches(sub2(a, b), pack_rn(__fsub_rn(a1, b1), __fsub_rn(a0, b0)));
         c_mul += mismatches(mul2(a, b), pack_rn(product_round_to_odd(a1, b1), product_round_to_odd(a0, b0)));
         c_div += mismatches(div2(a, b), div2_ieee(a, b));
+        {
+            // the branch-free quotient of the lean chain: a lane it does not flag must already be right,
+            // for every divisor it admits (NaN, Inf, normal up to 2^126)
+            uint32_t flag = 0u;
+            const bf2 q = div2_normal_divisor_deferred(a, b, flag), ref = div2_ieee(a, b);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const uint32_t d = (b >> (16 * h)) & 0x7FFFu, e = d >> 7;
+                const bool admitted = e == 0xFFu || (e >= 1u && d <= 0x7E80u);
+                const bool flagged = ((flag >> (16 * h)) & 0xFFFFu) != 0u;
+                if (admitted && !flagged && !same_or_both_nan((q >> (16 * h)) & 0xFFFFu, (ref >> (16 * h)) & 0xFFFFu)) ++c_div;
+            }
+        }
         // scalar-divisor route: divisors are the positive normal values up to 1 (bias corrections live there)
         if (b16 >= 0x0080u && b16 + 1u <= 0x3F80u) {
             const double d0 = static_cast<double>(b0), d1 = static_cast<double>(b1);
@@ -280,6 +293,17 @@ __global__ void __launch_bounds__(256) selftest_kernel(unsigned long long* count
         const uint32_t x = static_cast<uint32_t>(i) * 2u;
         const bf2 a = x | ((x + 1u) << 16);
         c_sqrt += mismatches(sqrt2(a), sqrt2_ieee(a));
+        // the branch-free root of the lean chain: unflagged lanes are right, except that a positive
+        // subnormal may come out as +0 (its contract)
+        uint32_t flag = 0u;
+        const bf2 s = sqrt2_flushing_deferred(a, flag), ref = sqrt2_ieee(a);
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t in = (a >> (16 * h)) & 0xFFFFu, got = (s >> (16 * h)) & 0xFFFFu;
+            const bool flagged = ((flag >> (16 * h)) & 0xFFFFu) != 0u;
+            const bool flushed = in >= 0x0001u && in <= 0x007Fu && got == 0u;
+            if (!flagged && !flushed && !same_or_both_nan(got, (ref >> (16 * h)) & 0xFFFFu)) ++c_sqrt;
+        }
     }
     unsigned long long v[6] = {c_add, c_sub, c_mul, c_div, c_sqrt, c_sdiv};
 #pragma unroll

@@ -158,24 +158,6 @@ __device__ __forceinline__ bf2 div2(bf2 a, bf2 b) {
 #endif
 }
 
-// a (/) b where the caller guarantees that b is NaN, Inf, or a normal number in [2^-126, 2^126]:
-// the reciprocal is then accurate and an overflowing quotient is correctly Inf, so only a tiny
-// (possibly tied) or NaN quotient needs the IEEE route.
-__device__ __forceinline__ bf2 div2_normal_divisor(bf2 a, bf2 b) {
-#ifdef COLLAGE_IEEE_DIV_SQRT
-    return div2_ieee(a, b);
-#else
-    const float a0 = lo_f32(a), a1 = hi_f32(a), b0 = lo_f32(b), b1 = hi_f32(b);
-    float q0 = __fmul_rn(a0, rcp_ftz(b0));
-    float q1 = __fmul_rn(a1, rcp_ftz(b1));
-    if (!(fabsf(q0) >= 0x1p-125f && fabsf(q1) >= 0x1p-125f)) {
-        if (!(fabsf(q0) >= 0x1p-125f)) q0 = div_out_of_range(a0, b0);
-        if (!(fabsf(q1) >= 0x1p-125f)) q1 = div_out_of_range(a1, b1);
-    }
-    return pack_rn(q1, q0);
-#endif
-}
-
 // a (/) s for a scalar 2^-100 <= s <= 1 whose reciprocal r was rounded to float on the host.
 // No range test is needed: |a*r| >= |a|, so a quotient can only be subnormal when a is, and then
 // both the float product and the exact quotient sit on grids (2^-149 and 1/(256*2^134)) that keep
@@ -213,17 +195,6 @@ __device__ __forceinline__ uint32_t less_than2(bf2 a, bf2 b) {
     asm("set.lt.u32.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
 }
-// sqrt(a) where the caller accepts +0 for a positive subnormal input (true root < 2^-63).  A negative
-// subnormal would be flushed to -0 instead of giving NaN, so any negative lane takes the careful route.
-__device__ __forceinline__ bf2 sqrt2_flushing(bf2 a) {
-#ifdef COLLAGE_IEEE_DIV_SQRT
-    return sqrt2_ieee(a);
-#else
-    if (less_than2(a, 0u)) return sqrt2(a);
-    return pack_rn(sqrt_ftz(hi_f32(a)), sqrt_ftz(lo_f32(a)));
-#endif
-}
-
 // ---- deferred forms: no branch; a lane the fast route cannot answer sets bits in `suspect`, and
 // the caller recomputes the whole vector by the careful routes when any bit is set ---------------
 __device__ __forceinline__ uint32_t less_equal2(bf2 a, bf2 b) {
@@ -242,10 +213,12 @@ __device__ __forceinline__ uint32_t equal2(bf2 a, bf2 b) {
     asm("set.eq.u32.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
 }
-// a (/) b under div2_normal_divisor's guarantee on b.  The rounded quotient is trusted unless its
-// magnitude is at most 2^-125 (the float product may then have been subnormal or tied) while the
-// numerator is not zero; a zero numerator gives the correctly signed zero (or NaN for a NaN
-// divisor) by the product alone, and a NaN product is a NaN quotient for every admitted divisor.
+// a (/) b where the caller guarantees that b is NaN, Inf, or a normal number in [2^-126, 2^126]:
+// the reciprocal is then accurate and an overflowing quotient is correctly Inf.  The rounded
+// quotient is trusted unless its magnitude is at most 2^-125 (the float product may then have
+// been subnormal or tied) while the numerator is not zero; a zero numerator gives the correctly
+// signed zero (or NaN for a NaN divisor) by the product alone, and a NaN product is a NaN quotient
+// for every admitted divisor.
 __device__ __forceinline__ bf2 div2_normal_divisor_deferred(bf2 a, bf2 b, uint32_t& suspect) {
 #ifdef COLLAGE_IEEE_DIV_SQRT
     return div2_ieee(a, b);
@@ -255,8 +228,9 @@ __device__ __forceinline__ bf2 div2_normal_divisor_deferred(bf2 a, bf2 b, uint32
     return q;
 #endif
 }
-// sqrt(a) under sqrt2_flushing's contract; a negative lane (NaN by IEEE, but -0 from the flushing
-// approximation when subnormal) marks the vector
+// sqrt(a) where the caller accepts +0 for a positive subnormal input (true root < 2^-63: the
+// approximation flushes it).  A negative lane (NaN by IEEE, but -0 from the flushing approximation
+// when subnormal) marks the vector.
 __device__ __forceinline__ bf2 sqrt2_flushing_deferred(bf2 a, uint32_t& suspect) {
 #ifdef COLLAGE_IEEE_DIV_SQRT
     return sqrt2_ieee(a);
