@@ -18,6 +18,10 @@
  *   - state tensors are updated in place; `grad` is read only;
  *   - calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL = default
  *     stream); the library never synchronises the device and never allocates on the step path;
+ *     collage_adamw_step, collage_adamw_step_multi and collage_adamw_step_fp32 only launch kernels,
+ *     so once a call of the same kind has run on the device (it sets per-device kernel attributes
+ *     the first time) they may be recorded by stream capture into a CUDA graph: the scalars of
+ *     the step are kernel arguments and are recorded with it;
  *   - errors are detected on the host BEFORE anything is launched and reported as a status
  *     code; nothing is thrown across the boundary; there is no CPU fallback: a device that is
  *     not compute capability 10.x yields COLLAGE_ERR_ARCH;

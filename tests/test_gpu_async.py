@@ -72,3 +72,92 @@ def test_two_streams_step_different_tensors_at_the_same_time():
     edq_close(e1.read(), want_big)
     edq_close(e2.read(), want_small)
     assert B.pipeline_fault() == 0
+
+
+@pytest.mark.parametrize("api", ["flat", "multi"])
+def test_steps_recorded_into_a_cuda_graph_replay_bit_identically(api):
+    # the step only launches kernels on the given stream (no allocation, no synchronisation, no host round trip),
+    # so three consecutive steps can be recorded once and replayed: same bits as the oracle, twice
+    n, hyp, strategy = 300_011, W.HYPERS, 2
+    st0 = oracle_state(W.bits(W.flat_weights(n, 74)), strategy)
+    grads = [W.bits(W.flat_grads(n, 74, t)) for t in (1, 2, 3)]
+    dev = {k: W.from_bits(v, "cuda") for k, v in st0.items()}
+    gdev = [W.from_bits(g, "cuda") for g in grads]
+    e = EdqBuffers()
+    plans = [B.plan_create([(dev["x_hi"], dev["x_lo"], dev["m"], dev["v_hi"], dev["v_lo"], g, n)]) for g in gdev] if api == "multi" else None
+
+    def enqueue(stream):
+        for t in (1, 2, 3):
+            if api == "multi":
+                B.adamw_step_multi(plans[t - 1], e.hyper(hyp), t, strategy, stream)
+            else:
+                B.adamw_step(dev["x_hi"], dev["x_lo"], dev["m"], dev["v_hi"], dev["v_lo"], gdev[t - 1], n, e.hyper(hyp), t, strategy, stream)
+
+    def restore():
+        for k, v in st0.items():
+            dev[k].copy_(W.from_bits(v, "cuda"))
+        torch.cuda.synchronize()
+
+    side = torch.cuda.Stream()
+    enqueue(side)                                   # first use: per-device kernel attributes are set outside the recording
+    side.synchronize()
+    restore()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        enqueue(side)
+    want = {k: v.copy() for k, v in st0.items()}
+    for t in (1, 2, 3):
+        sums = oracle_step(want, grads[t - 1], t, strategy, hyp)
+    for rep in range(2):
+        restore()
+        graph.replay()
+        torch.cuda.synchronize()
+        _check(dev, want, f"graph replay {rep} ({api})")
+        edq_close(e.read(), sums)
+    if plans:
+        for p in plans:
+            B.plan_destroy(p)
+    assert B.pipeline_fault() == 0
+
+
+def test_fp32_comparator_step_recorded_into_a_cuda_graph():
+    import oracle
+    from conftest import bits_to_f64
+    n, hyp = 200_003, W.HYPERS
+    theta0 = W.bits(W.flat_weights(n, 75))
+    grads = [W.bits(W.flat_grads(n, 75, t)) for t in (1, 2)]
+    d_theta, d_master = W.from_bits(theta0, "cuda"), torch.from_numpy(bits_to_f64(theta0).astype(np.float32)).cuda()
+    d_m, d_v = torch.zeros(n, dtype=torch.float32, device="cuda"), torch.zeros(n, dtype=torch.float32, device="cuda")
+    gdev = [W.from_bits(g, "cuda") for g in grads]
+    e = EdqBuffers()
+
+    def enqueue(stream):
+        for t in (1, 2):
+            B.adamw_step_fp32(d_theta, d_master, d_m, d_v, gdev[t - 1], n, e.hyper(hyp), t, stream)
+
+    def restore():
+        d_theta.copy_(W.from_bits(theta0, "cuda"))
+        d_master.copy_(torch.from_numpy(bits_to_f64(theta0).astype(np.float32)).cuda())
+        d_m.zero_()
+        d_v.zero_()
+        torch.cuda.synchronize()
+
+    side = torch.cuda.Stream()
+    enqueue(side)
+    side.synchronize()
+    restore()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        enqueue(side)
+    theta, master = theta0.copy(), bits_to_f64(theta0).astype(np.float32)
+    m, v = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    for t in (1, 2):
+        want = oracle.adamw_fp32_step(theta, master, m, v, grads[t - 1], step=t, **hyp)
+    restore()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert np.array_equal(W.bits(d_theta), theta)
+    assert np.array_equal(d_master.cpu().numpy().view(np.uint32), master.view(np.uint32))
+    assert np.array_equal(d_v.cpu().numpy().view(np.uint32), v.view(np.uint32))
+    edq_close(e.read(), want)
+    assert B.pipeline_fault() == 0
