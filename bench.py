@@ -311,9 +311,30 @@ def run_size_sweep(args):
             torch.cuda.synchronize()
             ms = e0.elapsed_time(e1) / iters
             gbs = n * BYTES_PER_PARAM[strategy] / (ms * 1e-3) / 1e9
-            print(json.dumps({"n": n, "strategy": name, "us_per_step": ms * 1e3, "params_per_sec": n / (ms * 1e-3),
-                              "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak, "frac_of_nominal_8TBps": gbs / 8000.0,
-                              "buffer_sets": sets, "launches_per_step": 2}), flush=True)
+            line = {"n": n, "strategy": name, "us_per_step": ms * 1e3, "params_per_sec": n / (ms * 1e-3),
+                    "hbm_gbs": gbs, "frac_of_measured_peak": gbs / peak, "frac_of_nominal_8TBps": gbs / 8000.0,
+                    "buffer_sets": sets, "launches_per_step": 2}
+            if p <= 11:
+                # the same steps recorded once into a CUDA graph and replayed: no per-launch host cost
+                side = torch.cuda.Stream()
+                side.wait_stream(stream)
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=side):
+                    for i in range(iters):
+                        B.adamw_step(*bufs[i % sets], n, h, 4 + i, strategy, side)
+                graph.replay()
+                torch.cuda.synchronize()
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record(stream)
+                for _ in range(3):
+                    graph.replay()
+                g1.record(stream)
+                torch.cuda.synchronize()
+                gms = g0.elapsed_time(g1) / (3 * iters)
+                line["us_per_step_graph"] = gms * 1e3
+                line["hbm_gbs_graph"] = n * BYTES_PER_PARAM[strategy] / (gms * 1e-3) / 1e9
+                del graph
+            print(json.dumps(line), flush=True)
             del bufs
             torch.cuda.empty_cache()
 
