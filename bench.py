@@ -404,9 +404,20 @@ def run_cpu_baseline(W, seconds=15.0, threads=None):
         el = time.perf_counter() - t0
         if el >= seconds or t >= 200:
             break
+    # one thread, on a 2^21-parameter piece of the same arrays (a few seconds)
+    n1 = 1 << 21
+    one = [a[:n1].copy() for a in st]
+    t1, s0 = 0, time.perf_counter()
+    while True:
+        t1 += 1
+        oracle.adamw_step(one[0], one[1], one[2], one[3], one[4], g[:n1].copy(), step=t + t1, strategy=STRATEGY, threads=1, **W.HYPERS)
+        e1 = time.perf_counter() - s0
+        if e1 >= 3.0 or t1 >= 50:
+            break
     return {"value": done / el, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": f"{t} Collage-plus steps over the first {n} parameters of the workload's embedding tensor "
-                      f"({el:.1f} s)"}
+                      f"({el:.1f} s)",
+            "value_one_thread": n1 * t1 / e1, "sample_one_thread": f"{t1} steps over {n1} parameters ({e1:.1f} s)"}
 
 
 def run_reference(args):
