@@ -299,6 +299,13 @@ collage_status_t collage_edq_static(const void* old_hi, const void* old_lo, cons
  * checkpoints, not per step.  Errors: ERR_NULL, ERR_CUDA. */
 collage_status_t collage_pipeline_fault(uint32_t* out_host);
 
+/* Exercises the give-up path of those waits without any fault: launches one warp that waits on a
+ * barrier nothing completes, bounded by about `limit_ms` milliseconds (1..1000, counted in SM
+ * cycles at 2 GHz).  The wait runs out, the kernel returns normally, and the next
+ * collage_pipeline_fault reports the code 100.  The device and the library stay usable.
+ * Asynchronous on `stream`.  Errors: ERR_ARG (limit out of range), ERR_ARCH, ERR_CUDA. */
+collage_status_t collage_wait_timeout_selftest(uint32_t limit_ms, void* stream);
+
 /* Exhaustive self test of the arithmetic the kernels rely on, on the current device (Section 3.1's
  * model: one rounding to nearest-even per operation).  Compares, for EVERY pair of bfloat16 bit
  * patterns (2^32 pairs; 2^16 values for the root), the realisation used in the kernels with a

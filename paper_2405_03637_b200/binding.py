@@ -24,7 +24,7 @@ EXPORTS = (
     "collage_plan_num_chunks", "collage_plan_set_replicas", "collage_plan_workspace_bytes", "collage_adamw_step_multi_per_tensor",
     "collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_grow",
     "collage_scaling", "collage_mul", "collage_renormalize", "collage_rounded_op", "collage_edq",
-    "collage_selftest", "collage_pipeline_fault", "collage_edq_static",
+    "collage_selftest", "collage_pipeline_fault", "collage_edq_static", "collage_wait_timeout_selftest",
 )
 
 
@@ -97,6 +97,7 @@ def lib() -> ctypes.CDLL:
         L.collage_edq_static.argtypes = [vp, vp, vp, vp, vp, u64, vp, vp]
         L.collage_selftest.argtypes = [ctypes.POINTER(ctypes.c_uint64), vp]
         L.collage_pipeline_fault.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
+        L.collage_wait_timeout_selftest.argtypes = [ctypes.c_uint32, ctypes.c_void_p]
         _lib = L
     return _lib
 
@@ -266,6 +267,10 @@ def pipeline_fault() -> int:
     out = ctypes.c_uint32(0)
     _check(lib().collage_pipeline_fault(ctypes.byref(out)), "collage_pipeline_fault")
     return int(out.value)
+
+
+def wait_timeout_selftest(limit_ms: int, stream=None):
+    _check(lib().collage_wait_timeout_selftest(limit_ms, _ptr(stream)), "collage_wait_timeout_selftest")
 
 
 def read_edq(edq_dev) -> dict:

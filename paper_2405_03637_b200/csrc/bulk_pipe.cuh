@@ -31,16 +31,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after ~4e9 cycles (about two seconds) and records in *fault_word which
-// wait failed (1 + who; the first failure wins).  The caller leaves its loops when this returns false.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int who, unsigned int* fault_word) {
+// Bounded wait: gives up after `limit` cycles (by default ~4e9, about two seconds) and records in
+// *fault_word which wait failed (1 + who; the first failure wins).  The caller leaves its loops
+// when this returns false.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int who, unsigned int* fault_word,
+                                          long long limit = 4000000000LL) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > 4000000000LL) {
+        if (clock64() - t0 > limit) {
             atomicCAS(fault_word, 0u, who + 1u);
             return false;
         }

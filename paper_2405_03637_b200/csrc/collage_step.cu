@@ -970,6 +970,30 @@ collage_status_t collage_pipeline_fault(uint32_t* out_host) {
     return COLLAGE_OK;
 }
 
+// ---- the give-up path of the bounded waits, exercised without a fault ---------------------------
+namespace collage {
+// One warp waits on a barrier that nothing completes, with a short bound; the wait runs out, the
+// code 100 goes to the fault word and the kernel returns in the ordinary way.
+__global__ void __launch_bounds__(32) wait_timeout_kernel(long long limit_cycles) {
+    __shared__ alignas(8) uint64_t bar;
+    if (threadIdx.x == 0) {
+        pipe::mbar_init(&bar, 1);
+        pipe::mbar_init_fence();
+    }
+    __syncwarp();
+    (void)__all_sync(0xFFFFFFFFu, pipe::mbar_wait(&bar, 0u, 99u, &g_pipeline_fault, limit_cycles));
+}
+}  // namespace collage
+
+collage_status_t collage_wait_timeout_selftest(uint32_t limit_ms, void* stream) {
+    if (limit_ms == 0 || limit_ms > 1000) return COLLAGE_ERR_ARG;
+    DeviceInfo dev;
+    const collage_status_t st = current_device(&dev);
+    if (st != COLLAGE_OK) return st;
+    wait_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<long long>(limit_ms) * 2000000LL);
+    return cudaGetLastError() == cudaSuccess ? COLLAGE_OK : COLLAGE_ERR_CUDA;
+}
+
 // ---- state in host memory: staged step -------------------------------------------------------
 
 namespace {

@@ -161,3 +161,33 @@ def test_fp32_comparator_step_recorded_into_a_cuda_graph():
     assert np.array_equal(d_v.cpu().numpy().view(np.uint32), v.view(np.uint32))
     edq_close(e.read(), want)
     assert B.pipeline_fault() == 0
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_device_stays_usable():
+    # the give-up path of the pipeline's bounded barrier waits, made on purpose with a barrier that nothing
+    # completes and a 20 ms bound: the kernel returns normally, the code is reported once, work goes on
+    assert B.pipeline_fault() == 0
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    B.wait_timeout_selftest(20)
+    t1.record()
+    torch.cuda.synchronize()
+    assert 5.0 < t0.elapsed_time(t1) < 500.0          # bounded: tens of milliseconds, not seconds
+    assert B.pipeline_fault() == 100
+    assert B.pipeline_fault() == 0                    # reading clears the word
+    with pytest.raises(B.CollageError):
+        B.wait_timeout_selftest(0)
+    with pytest.raises(B.CollageError):
+        B.wait_timeout_selftest(5000)
+    n, hyp = 20_011, W.HYPERS
+    st = oracle_state(W.bits(W.flat_weights(n, 76)), 2)
+    dev = {k: W.from_bits(v, "cuda") for k, v in st.items()}
+    g = W.bits(W.flat_grads(n, 76, 1))
+    e = EdqBuffers()
+    B.adamw_step(dev["x_hi"], dev["x_lo"], dev["m"], dev["v_hi"], dev["v_lo"], W.from_bits(g, "cuda"), n, e.hyper(hyp), 1, 2)
+    torch.cuda.synchronize()
+    want = oracle_step(st, g, 1, 2, hyp)
+    _check(dev, st, "step after a reported timeout")
+    edq_close(e.read(), want)
+    assert B.pipeline_fault() == 0
