@@ -33,6 +33,14 @@ WORKLOAD = "llama7b_shaped_291_tensors_collage_plus_with_edq"
 NCU_TRAFFIC_BYTES_PER_PARAM = (3.146235e9 + 2.567421e9) / 262_148_096
 
 
+def host_threads():
+    """Cores this process may run on: the oracle's thread count (a launcher's OMP_NUM_THREADS=1 does not apply)."""
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
 def measured_hbm_peak():
     f = ROOT / "MEASURED_PEAKS.json"
     if f.exists():
@@ -391,7 +399,7 @@ def run_cpu_baseline(W, seconds=15.0, threads=None):
     """The oracle as it stands on this machine's cores, on a bounded slice of the same workload."""
     import numpy as np
     import oracle
-    threads = threads or oracle.max_threads()
+    threads = threads or host_threads()
     n = 1 << 24
     theta = W.bits(W.normal_bf16(n, 0.02, 300_000))
     g = W.bits(W.normal_bf16(n, 1e-3, 350_000))
@@ -427,7 +435,7 @@ def run_reference(args):
     import numpy as np
     import oracle
     from paper_2405_03637_b200 import workloads as W
-    threads = oracle.max_threads()
+    threads = host_threads()
     n = 1 << 23
     theta = W.bits(W.normal_bf16(n, 0.02, 300_000))
     g = W.bits(W.normal_bf16(n, 1e-3, 350_000))
