@@ -13,6 +13,10 @@
 // Tiles that cannot be bulk-copied (tensor not 16-byte aligned, or the ragged last tile of a
 // tensor) flow through the same barriers but are processed straight from global memory.
 // Every wait is bounded: after ~2 s a thread records a fault in g_pipeline_fault and leaves.
+//
+// On the host-validated lean chain (FAST) a consumer runs the branch-free compute_vec_fast on its
+// 8 parameters; a vector with a lane that chain cannot answer is repeated in place, from the tile
+// that still holds its inputs, by the out-of-line careful_vector_in_tile.
 #pragma once
 #include "bulk_pipe.cuh"
 #include "mcf_device.cuh"
