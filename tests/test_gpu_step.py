@@ -321,3 +321,46 @@ def test_sparse_rare_lanes_between_ordinary_ones_keep_state_edq_and_lost_exact(s
     dev = _device_state(st)
     lost = [step(t)["lost"] for t in (2, 3, 4)]
     assert min(lost) > 0        # the poked parameters do lose updates, so the exact count is exercised
+
+
+HYPER_SWEEP = [
+    # lr, beta1, beta2, eps, weight_decay, step
+    (1e-4, 0.9, 0.999, 1e-8, 0.1, 1),
+    (1e-4, 0.9, 0.999, 1e-8, 0.1, 1_000_000),        # bias corrections round to 1
+    (1e-4, 0.9, 0.999, 1e-8, 0.1, 10 ** 9),
+    (0.0, 0.9, 0.999, 1e-8, 0.1, 3),                 # zero learning rate: every update is a signed zero
+    (1.0, 0.0, 0.5, 1e-8, 0.0, 2),                   # no momentum, fast second moment, huge steps
+    (3e-3, 0.5, 0.95, 1e-6, 0.5, 7),
+    (1e-5, 0.99, 0.9999, 1e-10, 0.01, 1000),
+    (6e-4, 0.9, 0.95, 1e-5, 0.1, 50),
+    (1e-2, 0.999, 0.9999, 1e-3, 1.0, 12345),
+    (2.5e-4, 0.8, 0.0, 1.0, 0.0, 4),                 # beta2 = 0: v is the last squared gradient; eps = 1
+]
+
+
+@pytest.mark.parametrize("strategy", [0, 1, 2, 3])
+def test_hyper_parameter_and_step_sweep(strategy):
+    # one step from a mid-training state for every row of the sweep: scalars derived on both sides independently
+    n = 70_001
+    rng = np.random.default_rng(40 + strategy)
+    for lr, b1, b2, eps, wd, t in HYPER_SWEEP:
+        hyp = dict(lr=lr, beta1=b1, beta2=b2, eps=eps, weight_decay=wd)
+        st = oracle_state(W.bits(W.flat_weights(n, 90)), strategy)
+        st["m"] = W.bits(W.normal_bf16(n, 1e-3, 91))
+        v = W.normal_bf16(n, 1e-3, 92).float().square().to(torch.bfloat16)
+        st["v_hi"] = W.bits(v)
+        if st["x_lo"] is not None:
+            st["x_lo"] = W.bits(W.normal_bf16(n, 2e-5, 93))
+        if st["v_lo"] is not None:              # a second component well below the first, either sign
+            st["v_lo"] = W.bits((v.float() * 1.5e-3 * torch.sign(W.normal_bf16(n, 1.0, 94).float())).to(torch.bfloat16))
+        g = W.bits(W.flat_grads(n, 90, 1))
+        g[rng.random(n) < 0.02] = 0
+        dev = _device_state(st)
+        e = EdqBuffers()
+        G = Guarded(g)
+        B.adamw_step(_t(dev["x_hi"]), _t(dev["x_lo"]), _t(dev["m"]), _t(dev["v_hi"]), _t(dev["v_lo"]), G.t, n,
+                     e.hyper(hyp), t, strategy)
+        torch.cuda.synchronize()
+        want = oracle_step(st, g, t, strategy, hyp)
+        _compare(dev, st, f"hypers {hyp} step {t} strategy {strategy}")
+        edq_close(e.read(), want)
