@@ -78,3 +78,30 @@ def test_fp32_comparator_argument_checks():
     assert err.value.status == B.ERR_ARG
     B.adamw_step_fp32(th, None, m, v, g, 0, h, 1)
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("with_master", [True, False])
+def test_fp32_comparator_over_a_sweep_of_hyper_parameters(with_master):
+    n = 30_011
+    sweep = [(1e-4, 0.9, 0.999, 1e-8, 0.1, 1_000_000), (0.0, 0.9, 0.999, 1e-8, 0.1, 3), (1.0, 0.0, 0.5, 1e-8, 0.0, 2),
+             (3e-3, 0.5, 0.95, 1e-6, 0.5, 7), (1e-2, 0.999, 0.9999, 1e-3, 1.0, 12345)]
+    for lr, b1, b2, eps, wd, t0 in sweep:
+        hyp = dict(lr=lr, beta1=b1, beta2=b2, eps=eps, weight_decay=wd)
+        theta = W.bits(W.flat_weights(n, 82))
+        master = bits_to_f64(theta).astype(np.float32) if with_master else None
+        m, v = np.zeros(n, np.float32), np.zeros(n, np.float32)
+        d_theta = W.from_bits(theta, "cuda")
+        d_m, d_v = torch.zeros(n, device="cuda"), torch.zeros(n, device="cuda")
+        d_w = torch.from_numpy(master).cuda() if with_master else None
+        e = EdqBuffers()
+        for t in (t0, t0 + 1, t0 + 2):
+            g = W.bits(W.flat_grads(n, 83, t % 1000))
+            B.adamw_step_fp32(d_theta, d_w, d_m, d_v, W.from_bits(g, "cuda"), n, e.hyper(hyp), t)
+            torch.cuda.synchronize()
+            want = oracle.adamw_fp32_step(theta, master, m, v, g, step=t, **hyp)
+            assert np.array_equal(W.bits(d_theta), theta), f"{hyp} theta step {t}"
+            assert np.array_equal(d_m.cpu().numpy().view(np.uint32), m.view(np.uint32)), f"{hyp} m step {t}"
+            assert np.array_equal(d_v.cpu().numpy().view(np.uint32), v.view(np.uint32)), f"{hyp} v step {t}"
+            if with_master:
+                assert np.array_equal(d_w.cpu().numpy().view(np.uint32), master.view(np.uint32)), f"{hyp} master step {t}"
+            edq_close(e.read(), want)

@@ -114,3 +114,45 @@ def test_float_arithmetic_in_registers_variant_bitwise(n, misalign, flags):
             assert dev[k].guards_intact()
         edq_close(e.read(), want)
     assert B.pipeline_fault() == 0
+
+
+VARIANT_HYPERS = [
+    # lr, beta1, beta2, eps, weight_decay, step
+    (1e-4, 0.9, 0.999, 1e-8, 0.1, 1_000_000),
+    (0.0, 0.9, 0.999, 1e-8, 0.1, 3),
+    (1.0, 0.0, 0.5, 1e-8, 0.0, 2),
+    (3e-3, 0.5, 0.95, 1e-6, 0.5, 7),
+    (1e-2, 0.999, 0.9999, 1e-3, 1.0, 12345),
+]
+
+
+@pytest.mark.parametrize("strategy,flags", [(1, B.FLAG_TWOSUM_GROW), (2, B.FLAG_TWOSUM_GROW), (2, B.FLAG_DECAY_BY_GROW),
+                                            (2, B.FLAG_TWOSUM_GROW | B.FLAG_DECAY_BY_GROW | B.FLAG_EPS_INSIDE_SQRT),
+                                            (0, B.FLAG_DECAY_BY_GROW), (4, 0)])
+def test_variants_over_a_sweep_of_hyper_parameters(strategy, flags):
+    # three steps from zero moments for every row: the flag paths and the register variant derive their scalars
+    # from the same host code as the default path, the oracle derives them on its own
+    n = 30_011
+    for lr, b1, b2, eps, wd, t0 in VARIANT_HYPERS:
+        hyp = dict(lr=lr, beta1=b1, beta2=b2, eps=eps, weight_decay=wd)
+        theta = W.bits(W.flat_weights(n, 95))
+        z = lambda: np.zeros(n, np.uint16)
+        st = dict(x_hi=theta.copy(), x_lo=z() if strategy else None, m=z(), v_hi=z(), v_lo=z() if strategy in (2, 4) else None)
+        dev = {k: (Guarded(v) if v is not None else None) for k, v in st.items()}
+        ptr = lambda k: dev[k].t if dev[k] is not None else None
+        e = EdqBuffers()
+        for t in (t0, t0 + 1, t0 + 2):
+            g = W.bits(W.flat_grads(n, 96, t % 1000))
+            G = Guarded(g)
+            B.adamw_step(ptr("x_hi"), ptr("x_lo"), ptr("m"), ptr("v_hi"), ptr("v_lo"), G.t, n, e.hyper(hyp, flags), t, strategy)
+            torch.cuda.synchronize()
+            if strategy == 4:
+                want = oracle.adamw_fp32_register_step(st["x_hi"], st["x_lo"], st["m"], st["v_hi"], st["v_lo"], g, step=t,
+                                                       flags=flags, **hyp)
+            else:
+                want, _ = oracle.adamw_step(st["x_hi"], st["x_lo"], st["m"], st["v_hi"], st["v_lo"], g, step=t,
+                                            strategy=strategy, flags=flags, **hyp)
+            for k in KEYS:
+                if st[k] is not None:
+                    assert_same_bits(dev[k].bits(), st[k], f"{hyp} step {t} strategy {strategy} flags {flags} {k}")
+            edq_close(e.read(), want)
