@@ -351,6 +351,10 @@ __global__ void __launch_bounds__(256) edq_finalize_kernel(const EdqPartial* par
                                                            collage_edq_t* out, int accumulate) {
     __shared__ double s_dot[256], s_sq[256];
     __shared__ unsigned long long s_lost[256];
+    // When launched with programmatic stream serialisation this block may already be resident while
+    // the step kernel runs: wait here until that kernel has completed and its partials are visible.
+    // (A no-op after an ordinary launch.)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     double d = 0.0, q = 0.0;
     unsigned long long l = 0;
     for (int i = threadIdx.x; i < count; i += 256) {
@@ -445,6 +449,27 @@ __global__ void __launch_bounds__(32) edq_sum_records_kernel(const collage_edq_t
 void launch_edq_finalize(const EdqPartial* partials, int count, uint64_t n, collage_edq_t* out, cudaStream_t stream,
                          bool accumulate) {
     edq_finalize_kernel<<<1, 256, 0, stream>>>(partials, count, n, out, accumulate ? 1 : 0);
+}
+
+// The same behind a step kernel that has issued griddepcontrol.launch_dependents: the launch is
+// allowed to start before that kernel ends (its first instruction waits for it), which takes the
+// launch latency of this small kernel off the end of every step.
+void launch_edq_finalize_overlapped(const EdqPartial* partials, int count, uint64_t n, collage_edq_t* out,
+                                    cudaStream_t stream, bool accumulate) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, edq_finalize_kernel, partials, count, n, out, accumulate ? 1 : 0) != cudaSuccess) {
+        (void)cudaGetLastError();
+        edq_finalize_kernel<<<1, 256, 0, stream>>>(partials, count, n, out, accumulate ? 1 : 0);
+    }
 }
 
 // ---------------------------------------------------------------- host side ---
@@ -722,8 +747,8 @@ collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi,
                     dev.sm_count, cs, &grid) != cudaSuccess)
         return COLLAGE_ERR_CUDA;
     if (edq) {
-        launch_edq_finalize(static_cast<EdqPartial*>(hyper->workspace), grid, n,
-                            static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
+        launch_edq_finalize_overlapped(static_cast<EdqPartial*>(hyper->workspace), grid, n,
+                                       static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
         if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
     return COLLAGE_OK;
@@ -849,7 +874,7 @@ collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const coll
         if (dispatch_step<false>(p, strategy, edq, dev.sm_count, cs, &grid) != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
     if (edq) {
-        launch_edq_finalize(p.partials, grid, plan->num_elements, static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
+        launch_edq_finalize_overlapped(p.partials, grid, plan->num_elements, static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
         if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
     return COLLAGE_OK;
@@ -1089,7 +1114,7 @@ collage_status_t collage_adamw_step_host(void* x_hi, void* x_lo, void* m, void* 
                                 v_lo ? dev_array(b, 4) : nullptr, dev_array(b, 5), len, k, strategy, edq, partials,
                                 dev.sm_count, cs, &grid));
         if (edq) {
-            launch_edq_finalize(partials, grid, len, record, cs, true);
+            launch_edq_finalize_overlapped(partials, grid, len, record, cs, true);
             COLLAGE_TRY(cudaGetLastError());
         }
         COLLAGE_TRY(cudaEventRecord(c->computed[b], cs));

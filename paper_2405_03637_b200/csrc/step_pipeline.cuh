@@ -74,6 +74,8 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
     using Smem = PipeSmem<CONSUMERS, VPT, STAGES, STRATEGY>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
 
+    // the small kernel that sums the EDQ partials may be launched now; it waits for this grid to end
+    if (EDQ && !PER_CHUNK) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const bool is_producer = threadIdx.x >= CONSUMERS;
     if (threadIdx.x == 0) {
 #pragma unroll
