@@ -202,3 +202,57 @@ def test_theta_replicas_are_written_by_the_step_itself(strategy):
     assert all(np.array_equal(b, rep[-1].bits()) for b, rep in zip(before, reps))
     assert B.pipeline_fault() == 0
     B.plan_destroy(plan)
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_sharded_step_of_emulated_ranks_gathers_theta_everywhere(world):
+    # ZeRO-1-style ownership on one device: every "rank" keeps its own full copy of theta (what its forward
+    # pass would read) and the optimizer state of its slice only; its step writes the new theta of the slice
+    # into every rank's copy.  The ranks' kernels do not wait on one another, so running them one after the
+    # other is the same computation.  Afterwards every copy equals the oracle's theta of the unsharded step,
+    # and the summed EDQ records equal its global EDQ.
+    from paper_2405_03637_b200 import sharding as S
+    shapes = [("a", 70_001), ("b", 4096), ("c", 33_333), ("d", 8), ("e", 250_000)]
+    sizes = [n for _, n in shapes]
+    strategy, hyp = 2, W.HYPERS
+    theta = [W.bits(W.flat_weights(n, 300 + i)) for i, n in enumerate(sizes)]
+    copies = [[W.from_bits(t, "cuda") for t in theta] for _ in range(world)]          # theta as each rank sees it
+    full = [oracle_state(t, strategy) for t in theta]
+    parts = S.partition(sizes, world)
+    plans, states, grads_dev, edqs = [], [], [], []
+    for r in range(world):
+        z = lambda i: torch.zeros(sizes[i], dtype=torch.bfloat16, device="cuda")
+        # state tensors of full length for simplicity; the rank touches its ranges only
+        rows = [(copies[r][i], z(i), z(i), z(i), z(i), torch.zeros(sizes[i], dtype=torch.bfloat16, device="cuda"), sizes[i])
+                for i in range(len(sizes))]
+        mine = S.slice_rows(rows, parts[r])
+        plan = B.plan_create(mine)
+        peers = [copies[q] for q in range(world) if q != r]
+        B.plan_set_replicas(plan, S.replica_rows(peers, parts[r]))
+        plans.append(plan)
+        states.append(rows)
+        edqs.append(EdqBuffers())
+    for t in (1, 2, 3):
+        gbits = [W.bits(W.flat_grads(n, 400 + i, t)) for i, n in enumerate(sizes)]
+        for r in range(world):
+            for i in range(len(sizes)):
+                states[r][i][5].copy_(W.from_bits(gbits[i], "cuda"))
+        for r in range(world):
+            B.adamw_step_multi(plans[r], edqs[r].hyper(hyp), t, strategy)
+        torch.cuda.synchronize()
+        sums = np.zeros(4)                                  # dot, sumsq, (unused), lost of the unsharded step
+        for st, g in zip(full, gbits):
+            w = oracle_step(st, g, t, strategy, hyp)
+            sums += np.array([w["dot"], w["sumsq"], 0.0, w["lost"]])
+        for r in range(world):
+            for i in range(len(sizes)):
+                assert_same_bits(W.bits(copies[r][i]), full[i]["x_hi"], f"world {world} step {t}: theta copy of rank {r}, tensor {i}")
+        recs = [e.read() for e in edqs]
+        got = S.allreduce_edq(torch.tensor([sum(x["dot"] for x in recs), sum(x["sumsq"] for x in recs),
+                                            float(sum(x["lost"] for x in recs))], dtype=torch.float64))
+        assert sum(x["n"] for x in recs) == sum(sizes)
+        assert abs(got["dot"] - sums[0]) <= 1e-5 * abs(sums[0]) and abs(got["sumsq"] - sums[1]) <= 1e-5 * sums[1]
+        assert got["lost"] == int(sums[3])
+    for p in plans:
+        B.plan_destroy(p)
+    assert B.pipeline_fault() == 0
