@@ -67,10 +67,11 @@ def test_llama7b_full_size_launch_sampled_parity():
     torch.cuda.empty_cache()
 
 
-def test_llama7b_layout_one_layer_whole_arrays_and_edq():
-    # the same layout with one transformer layer (464 M parameters): every element and the global EDQ
+def test_llama7b_layout_four_layers_whole_arrays_and_edq():
+    # the same layout with four transformer layers (1.07 G parameters, 39 tensors): every element and the global EDQ
     dev = torch.device("cuda")
-    arrays, rows, n = bench.build_llama7b_state(torch, W, dev, seed=3, layers=1)
+    arrays, rows, n = bench.build_llama7b_state(torch, W, dev, seed=3, layers=4)
+    assert n == 262_148_096 + 4 * 202_383_360
     plan = B.plan_create(rows)
     e = EdqBuffers()
     st = {k: W.bits(arrays[k]) for k in KEYS}
