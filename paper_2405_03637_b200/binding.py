@@ -7,9 +7,12 @@ There is no fallback: if the shared library has not been built, loading raises.
 from __future__ import annotations
 
 import ctypes
+import os
 from pathlib import Path
 
-_LIB_PATH = Path(__file__).resolve().parent / "libcollage_b200.so"
+# the in-tree build, unless COLLAGE_B200_LIB names another build of the same sources (see build.py --out)
+_LIB_PATH = Path(os.environ["COLLAGE_B200_LIB"]).resolve() if os.environ.get("COLLAGE_B200_LIB") \
+    else Path(__file__).resolve().parent / "libcollage_b200.so"
 
 OK, ERR_NULL, ERR_ARG, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_WORKSPACE, ERR_LIMIT = range(8)
 BF16, LIGHT, PLUS, KAHAN, PLUS_FP32_REGISTERS = 0, 1, 2, 3, 4

@@ -1,6 +1,11 @@
 """Builds the CUDA library in-tree with nvcc for sm_100a (cross-compiles without a GPU).
 
-    python -m paper_2405_03637_b200.build [--force] [--verbose]
+    python -m paper_2405_03637_b200.build [--force] [--verbose] [--define NAME[=VALUE]]... [--out PATH]
+
+--define adds a preprocessor definition (the geometry constants COLLAGE_PIPE_* / COLLAGE_FP32_*, or
+COLLAGE_DATA_MOVEMENT_ONLY, which compiles the arithmetic out of the step kernel to measure what the
+copy pipeline alone sustains); such a build goes to --out, never over the in-tree library, and is
+loaded by pointing the environment variable COLLAGE_B200_LIB at it.
 
 The exactness of the error-free transforms depends on the flags below: no FMA contraction,
 no flush-to-zero, IEEE division and square root, never --use_fast_math.
@@ -29,20 +34,27 @@ def _newest_source_mtime() -> float:
     return max(f.stat().st_mtime for f in files)
 
 
-def build(force: bool = False, verbose: bool = False) -> Path:
-    if not force and LIB.exists() and LIB.stat().st_mtime >= _newest_source_mtime():
+def build(force: bool = False, verbose: bool = False, defines: tuple = (), out: Path | None = None) -> Path:
+    if defines and out is None:
+        raise ValueError("a build with extra definitions needs its own output path")
+    lib = Path(out) if out is not None else LIB
+    if out is None and not force and LIB.exists() and LIB.stat().st_mtime >= _newest_source_mtime():
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB.with_suffix(f".so.tmp{os.getpid()}")
-    cmd = [nvcc, *NVCC_FLAGS, *(["-Xptxas", "-v"] if verbose else []), "-o", str(tmp), *[str(CSRC / s) for s in SOURCES]]
+    tmp = lib.with_suffix(f".so.tmp{os.getpid()}")
+    cmd = [nvcc, *NVCC_FLAGS, *[f"-D{d}" for d in defines], *(["-Xptxas", "-v"] if verbose else []), "-o", str(tmp),
+           *[str(CSRC / s) for s in SOURCES]]
     proc = subprocess.run(cmd, capture_output=True, text=True)
     if verbose or proc.returncode:
         sys.stderr.write(proc.stdout + proc.stderr)
     if proc.returncode:
         raise RuntimeError("nvcc failed building the Collage CUDA library")
-    os.replace(tmp, LIB)
-    return LIB
+    os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    argv = sys.argv[1:]
+    defs = tuple(argv[i + 1] for i, a in enumerate(argv) if a == "--define" and i + 1 < len(argv))
+    outp = next((Path(argv[i + 1]) for i, a in enumerate(argv) if a == "--out" and i + 1 < len(argv)), None)
+    print(build(force="--force" in argv, verbose="--verbose" in argv, defines=defs, out=outp))

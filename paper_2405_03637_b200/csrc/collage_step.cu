@@ -132,6 +132,9 @@ struct Vec {
 template <int STRATEGY, bool EDQ, bool VARIANT = false>
 __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int valid, double& dot, double& sq,
                                             uint32_t& lost) {
+#ifdef COLLAGE_DATA_MOVEMENT_ONLY
+    return;     // measurement build: every array goes through the pipeline unchanged
+#endif
     uint32_t* th = reinterpret_cast<uint32_t*>(&s.th);
     uint32_t* dth = reinterpret_cast<uint32_t*>(&s.dth);
     uint32_t* m = reinterpret_cast<uint32_t*>(&s.m);
@@ -225,6 +228,9 @@ __device__ __forceinline__ void compute_vec(Vec& s, const StepScalars& k, int va
 template <int STRATEGY, bool EDQ, bool VARIANT = false>
 __device__ __forceinline__ uint32_t compute_vec_fast(Vec& s, const StepScalars& k, double& dot, double& sq, uint32_t& lost) {
     static_assert(STRATEGY != 4, "the register variant has no fast chain");
+#ifdef COLLAGE_DATA_MOVEMENT_ONLY
+    return 0u;  // measurement build: every array goes through the pipeline unchanged
+#endif
     uint32_t* th = reinterpret_cast<uint32_t*>(&s.th);
     uint32_t* dth = reinterpret_cast<uint32_t*>(&s.dth);
     uint32_t* m = reinterpret_cast<uint32_t*>(&s.m);
