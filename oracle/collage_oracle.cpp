@@ -213,6 +213,20 @@ inline pair16 grow_two_sum(pair16 xy, bf16 a) {
 
 struct edq_sums { double dot, sumsq; uint64_t lost; };
 
+// Is the effective update (theta' + dtheta') - (theta + dtheta) of Eq. 2 zero?  A yes/no decision taken
+// by floating point: it is evaluated in single precision, differences first, the precision in which the
+// device forms the same quantity, so that both sides decide alike on every input.  For normalised
+// expansions (|lo| <= ulp(hi)/2, which Grow maintains) the single-precision result is zero exactly when
+// the real number is: each difference of two bfloat16 values is either exact in single precision or so
+// large that the other difference cannot cancel it, and an IEEE addition of two non-zero numbers gives
+// zero only when they are opposite.  tests/test_oracle_step.py checks this against exact rationals.
+inline bool value_unchanged(bf16 hi_old, bf16 lo_old, bf16 hi_new, bf16 lo_new, bool pair) {
+    const float move_hi = static_cast<float>(widen(hi_new)) - static_cast<float>(widen(hi_old));
+    if (!pair) return move_hi == 0.0f;
+    const float move_lo = static_cast<float>(widen(lo_new)) - static_cast<float>(widen(lo_old));
+    return move_hi + move_lo == 0.0f;
+}
+
 // One parameter, one step of Algorithm 2 (lines 8-13), in the printed order.
 // Returns the bfloat16 update (line 12) and accumulates the EDQ sums
 // (Eq. 2 and Eq. 3) in double.
@@ -276,10 +290,10 @@ inline void step_one(bf16& th, bf16* dth, bf16& m, bf16& v, bf16* dv, bf16 g,
     const double d = widen(delta) + (split_decay ? widen(decay) : 0.0);      // intended update
     acc.dot += d * eff;
     acc.sumsq += d * d;
-    // lost arithmetic (Def. 3.2; "not updated", Figure 3 left): an update was intended and the stored
-    // parameter (every component, compared as values) is what it was
-    const bool unchanged = widen(th) == widen(th_old) && (!pair_value || widen(*dth) == widen(dth_old));
-    if (d != 0.0 && unchanged) acc.lost += 1;
+    // lost arithmetic (Def. 3.2; "not updated", Figure 3 left): an update was intended and the parameter
+    // did not move, i.e. the effective update of Eq. 2 is zero.  For an expansion the parameter is the
+    // value theta + dtheta: a Grow that re-splits the same value over other components has not updated it.
+    if (d != 0.0 && value_unchanged(th_old, dth_old, th, pair_value ? *dth : 0, pair_value)) acc.lost += 1;
     if (delta_out) *delta_out = delta;
 }
 
@@ -407,9 +421,8 @@ void oracle_edq(const uint16_t* old_hi, const uint16_t* old_lo, const uint16_t* 
         const double d = widen(delta[i]);
         tot.dot += d * eff;
         tot.sumsq += d * d;
-        const bool unchanged = widen(new_hi[i]) == widen(old_hi[i]) &&
-                               (!(old_lo && new_lo) || widen(new_lo[i]) == widen(old_lo[i]));
-        if (d != 0.0 && unchanged) tot.lost += 1;
+        const bool pair = old_lo && new_lo;
+        if (d != 0.0 && value_unchanged(old_hi[i], pair ? old_lo[i] : 0, new_hi[i], pair ? new_lo[i] : 0, pair)) tot.lost += 1;
     }
     sums_out[0] = tot.dot;
     sums_out[1] = tot.sumsq;
@@ -530,7 +543,7 @@ void oracle_adamw_fp32_register_step(uint16_t* x_hi, uint16_t* x_lo, uint16_t* m
         const uint16_t vh = round_to_bf16(static_cast<double>(v_new));
         const uint16_t vl = round_to_bf16(static_cast<double>(v_new - f(vh)));
         const double eff = (widen(th) - widen(x_hi[i])) + (widen(dth) - widen(x_lo[i]));
-        const bool unchanged = widen(th) == widen(x_hi[i]) && widen(dth) == widen(x_lo[i]);
+        const bool unchanged = value_unchanged(x_hi[i], x_lo[i], th, dth, true);
         x_hi[i] = th;
         x_lo[i] = dth;
         m[i] = round_to_bf16(static_cast<double>(m_new));

@@ -120,6 +120,23 @@ def scaling(v, a1, a2):
     return fast_two_sum(x, e)
 
 
+def value_unchanged(th_old, dth_old, th_new, dth_new) -> bool:
+    """Is the effective update of Eq. 2, (theta' + dtheta') - (theta + dtheta), exactly zero?"""
+    return decode(th_new) + decode(dth_new) == decode(th_old) + decode(dth_old)
+
+
+def components_unchanged(th_old, dth_old, th_new, dth_new) -> bool:
+    """The other candidate reading of "not updated": every stored component kept its value."""
+    return decode(th_new) == decode(th_old) and decode(dth_new) == decode(dth_old)
+
+
+def is_normalised(hi, lo) -> bool:
+    """|lo| <= ulp(hi)/2 (Def. 3.1 with 7 stored bits), the invariant Grow maintains."""
+    field = (hi >> 7) & 0xFF
+    ulp = TWO ** (max(field - 127, -126) - 7)
+    return abs(decode(lo)) <= ulp / 2
+
+
 def two_sum(a, b):
     x = add(a, b)
     bv = sub(x, a)

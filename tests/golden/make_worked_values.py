@@ -52,6 +52,27 @@ def main():
             th, dth, m, v, dv, d = R.adamw_element(th, dth, m, v, dv, g, sc, strategy, eps_inside=True)
             lines.append(f"trace2 strategy={strategy} t={t} g={g:04X} | th={th:04X} dth={dth:04X} m={m:04X} "
                          f"v={v:04X} dv={dv:04X} delta={d:04X}")
+    # "Not updated" (Figure 3, left; Def. 3.2) for a parameter held as an expansion: the effective update of
+    # Eq. 2 is zero, decided here on exact rationals.  `lost` is that decision; `components` says whether both
+    # stored bit patterns kept their value, a different reading that the cases marked "resplit" tell apart:
+    # Grow returns the same value split over other components.  Found by scanning normalised pairs in order.
+    picked = {"resplit": [], "kept": [], "moved": []}
+    for a in (0x35AB, 0xB5AB, 0x3480, 0xB6C0):
+        room = {"resplit": len(picked["resplit"]) + 5, "kept": len(picked["kept"]) + 2, "moved": len(picked["moved"]) + 2}
+        for hi in list(range(0x3EF8, 0x3F08)) + list(range(0xBF7C, 0xBF84)):
+            for lo in list(range(0x3A00, 0x3B81)) + list(range(0xBA00, 0xBB81)) + [0]:
+                if not R.is_normalised(hi, lo):
+                    continue
+                u, v = R.grow(hi, lo, a)
+                same_value = R.value_unchanged(hi, lo, u, v)
+                same_bits = R.components_unchanged(hi, lo, u, v)
+                kind = "resplit" if same_value and not same_bits else "kept" if same_value else "moved"
+                if len(picked[kind]) < room[kind] and (kind != "resplit" or R.is_normalised(u, v)):
+                    picked[kind].append((hi, lo, a, u, v, same_value, same_bits))
+    for kind in ("resplit", "kept", "moved"):
+        for k, (hi, lo, a, u, v, same_value, same_bits) in enumerate(picked[kind]):
+            lines.append(f"lost {kind} {k} | x={hi:04X} y={lo:04X} a={a:04X} u={u:04X} v={v:04X} "
+                         f"lost={int(same_value)} components={int(same_bits)}")
     (HERE / "worked_values.txt").write_text("\n".join(lines) + "\n")
 
 

@@ -308,3 +308,85 @@ def test_bytes_per_parameter_accounting():
         st = W.fresh_state(W.flat_weights(n, 0), s)
         sizes.append((sum(t.numel() * t.element_size() for t in st.arrays()) + n * 2) // n)   # + gradient
     assert sizes == want[:3]
+
+
+# ------------------------------------------------ "not updated" (Def. 3.2) ---
+
+def _lost_records():
+    out = []
+    for key, val in _records("worked_values.txt").items():
+        if key.startswith("lost "):
+            f = dict(p.split("=") for p in val.split())
+            out.append((key.split()[1], *(int(f[k], 16) for k in ("x", "y", "a", "u", "v")), int(f["lost"]), int(f["components"])))
+    return out
+
+
+def test_lost_counts_parameters_whose_value_did_not_move_worked_cases():
+    # Figure 3 (left) counts parameters that were "not updated"; Eq. 2 defines the effective update.  The worked
+    # cases come from exact rationals: Grow may hand back the same value split over other components
+    # ("resplit"): the parameter has not moved and is counted, although both stored patterns changed.
+    recs = _lost_records()
+    assert {r[0] for r in recs} == {"resplit", "kept", "moved"} and sum(r[0] == "resplit" for r in recs) >= 12
+    arr = lambda k: np.array([r[k] for r in recs], np.uint16)
+    x, y, a, u, v = (arr(k) for k in range(1, 6))
+    gu, gv = oracle.grow(x, y, a)
+    assert np.array_equal(gu, u) and np.array_equal(gv, v)
+    for i, r in enumerate(recs):
+        got = oracle.edq(x[i:i + 1], y[i:i + 1], u[i:i + 1], v[i:i + 1], a[i:i + 1])
+        assert got["lost"] == r[6], r
+        if r[0] == "resplit":
+            assert r[6] == 1 and r[7] == 0          # the component reading would say "updated" here
+            assert got["dot"] == 0.0                # and EDQ agrees that nothing was applied
+    assert oracle.edq(x, y, u, v, a)["lost"] == sum(r[6] for r in recs)
+    # an intended update of zero is never "lost", whatever the pair does
+    assert oracle.edq(x, y, u, v, np.zeros_like(a))["lost"] == 0
+
+
+def test_lost_decision_equals_exact_rationals_on_normalised_pairs():
+    # every normalised pair of a window around a binade edge, four updates: the oracle's yes/no per parameter
+    # equals the exact decision "theta' + dtheta' == theta + dtheta" on rationals
+    his = list(range(0x3EFC, 0x3F04)) + list(range(0xBF7E, 0xBF82)) + [0x0080, 0x0001, 0x7F00]
+    los = list(range(0x3A70, 0x3A90)) + list(range(0xBAF0, 0xBB02)) + [0x0000, 0x8000, 0x0001, 0x3680]
+    cases = [(h, l, a) for a in (0x35AB, 0xB5AB, 0xB6C0, 0x3B00) for h in his for l in los if R.is_normalised(h, l)]
+    x, y, a = (np.array(c, np.uint16) for c in zip(*cases))
+    u, v = oracle.grow(x, y, a)
+    n_resplit = 0
+    for i, (h, l, d) in enumerate(cases):
+        ru, rv = R.grow(h, l, d)
+        assert (int(u[i]), int(v[i])) == (ru, rv)
+        want = R.value_unchanged(h, l, ru, rv)
+        got = oracle.edq(x[i:i + 1], y[i:i + 1], u[i:i + 1], v[i:i + 1], a[i:i + 1])["lost"]
+        assert got == int(want), (hex(h), hex(l), hex(d))
+        n_resplit += want and not R.components_unchanged(h, l, ru, rv)
+    assert n_resplit > 20 and len(cases) > 1500
+
+
+@pytest.mark.parametrize("strategy", [0, 1, 2, 3])
+def test_step_lost_count_against_exact_rationals(strategy):
+    # the stress distributions (|theta| in [0.5, 4), updates mostly far below ulp/2), run until the second
+    # component saturates: the step's count equals the exact per-parameter decision on the arrays before/after
+    n = 1500
+    th = W.bits(W.stress_weights(n, 2))
+    st = _state(th.copy(), min(strategy, 2) if strategy != 3 else 1)
+    st = dict(st, v_lo=st["v_lo"] if strategy == 2 else None)
+    seen_lost = seen_resplit = 0
+    for t in range(1, 61):
+        g = W.bits(W.stress_grads(n, 2, t))
+        before = (st["x_hi"].copy(), st["x_lo"].copy() if st["x_lo"] is not None else None)
+        sums, d = _step(st, g, t, strategy, hyp=W.HYPERS_STRESS, want_delta=True)
+        if t % 10:
+            continue
+        want = 0
+        for i in range(n):
+            if R.decode(int(d[i])) == 0:
+                continue
+            if strategy in (1, 2):
+                same = R.value_unchanged(int(before[0][i]), int(before[1][i]), int(st["x_hi"][i]), int(st["x_lo"][i]))
+                seen_resplit += same and not R.components_unchanged(int(before[0][i]), int(before[1][i]),
+                                                                    int(st["x_hi"][i]), int(st["x_lo"][i]))
+            else:       # plain bfloat16 and Kahan: the parameter is theta alone
+                same = R.decode(int(before[0][i])) == R.decode(int(st["x_hi"][i]))
+            want += same
+        assert sums["lost"] == want, (strategy, t)
+        seen_lost += want
+    assert seen_lost > 0
