@@ -93,7 +93,9 @@ typedef struct collage_hyper {
  *   dot   = sum_i delta_i * eff_i        eff = (theta'+dtheta') - (theta+dtheta)   (Eq. 2)
  *   sumsq = sum_i delta_i^2              delta = the bfloat16 update of Algorithm 2 line 12
  *   edq   = dot / sqrt(sumsq), 0 if sumsq == 0
- *   lost  = #{i : delta_i != 0 and no component of the stored parameter changed} (Def. 3.2)
+ *   lost  = #{i : delta_i != 0 and eff_i == 0}: parameters that an update was meant for and that did not
+ *           move (Def. 3.2; "not updated", Figure 3 left).  For a pair the value theta + dtheta counts:
+ *           a Grow that re-splits the same value over other components has not updated it.
  * Products and 8-element partial sums are formed in float, everything above in double, in a
  * fixed order: the result is reproducible for a given launch geometry. */
 typedef struct collage_edq {

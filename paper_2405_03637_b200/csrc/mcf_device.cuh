@@ -423,38 +423,34 @@ struct EdqAcc {
 };
 
 // `d` is the intended update as two floats; the stored parameter is (th, dth) when HAS_LO, else th alone.
+// A parameter counts as lost (Definition 3.2; "not updated", Figure 3 left) when an update was intended
+// and the effective update e of Eq. 2 is zero: the value theta + dtheta did not move, whether or not
+// Grow re-split it over other components.  e is formed in float, differences first; for normalised
+// pairs it is zero exactly when the real number is (each difference of two bfloat16 values is exact in
+// float unless it is far too large for the other difference to cancel, and a float sum of two
+// non-zero numbers is zero only when they are opposite).
 template <bool HAS_LO>
 __device__ __forceinline__ void edq_pair_f(EdqAcc& acc, bf2 th_old, bf2 dth_old, bf2 th_new, bf2 dth_new, f32x2 d) {
-    const f32x2 o = widen2(th_old), n = widen2(th_new);
-    f32x2 e = sub_f32x2(n, o);
-    bool same0 = lo_of(n) == lo_of(o), same1 = hi_of(n) == hi_of(o);
-    if (HAS_LO) {
-        const f32x2 p = widen2(dth_old), q = widen2(dth_new);
-        e = add_f32x2(e, sub_f32x2(q, p));
-        same0 = same0 && lo_of(q) == lo_of(p);
-        same1 = same1 && hi_of(q) == hi_of(p);
-    }
+    f32x2 e = sub_f32x2(widen2(th_new), widen2(th_old));
+    if (HAS_LO) e = add_f32x2(e, sub_f32x2(widen2(dth_new), widen2(dth_old)));
     acc.dot = fma_f32x2(d, e, acc.dot);
     acc.sq = fma_f32x2(d, d, acc.sq);
-    acc.lost += (lo_of(d) != 0.0f && same0) ? 1u : 0u;
-    acc.lost += (hi_of(d) != 0.0f && same1) ? 1u : 0u;
+    acc.lost += (lo_of(d) != 0.0f && lo_of(e) == 0.0f) ? 1u : 0u;
+    acc.lost += (hi_of(d) != 0.0f && hi_of(e) == 0.0f) ? 1u : 0u;
 }
-// The same with the comparisons of Definition 3.2 done on the packed bfloat16 values (widening is
-// exact, so they decide as the float comparisons do: zeros of either sign are equal, NaN equals
-// nothing and differs from zero).  `asked` is the intended update as a bfloat16 pair, zero where
-// `d` is.  acc.lost collects the two halves as packed 16-bit counts: see edq_lost_packed.
+// The same with the two decisions taken on packed bfloat16 values.  `asked` is the intended update as
+// a bfloat16 pair, zero where `d` is.  e is rounded to bfloat16 only to be compared with zero: every
+// term is a multiple of 2^-133, so a non-zero e is at least the smallest bfloat16 subnormal and stays
+// non-zero, a NaN stays NaN (equal to nothing), and zeros of either sign compare equal.
+// acc.lost collects the two halves as packed 16-bit counts: see edq_lost_packed.
 template <bool HAS_LO>
 __device__ __forceinline__ void edq_pair_packed(EdqAcc& acc, bf2 th_old, bf2 dth_old, bf2 th_new, bf2 dth_new, f32x2 d,
                                                 bf2 asked) {
     f32x2 e = sub_f32x2(widen2(th_new), widen2(th_old));
-    uint32_t unchanged = equal2(th_new, th_old);
-    if (HAS_LO) {
-        e = add_f32x2(e, sub_f32x2(widen2(dth_new), widen2(dth_old)));
-        unchanged &= equal2(dth_new, dth_old);
-    }
+    if (HAS_LO) e = add_f32x2(e, sub_f32x2(widen2(dth_new), widen2(dth_old)));
     acc.dot = fma_f32x2(d, e, acc.dot);
     acc.sq = fma_f32x2(d, d, acc.sq);
-    acc.lost += unchanged & differs2(asked, 0u) & 0x00010001u;
+    acc.lost += equal2(pack_rn2(e), 0u) & differs2(asked, 0u) & 0x00010001u;
 }
 // the count held in packed form by edq_pair_packed (at most 65535 pairs between two calls)
 __device__ __forceinline__ uint32_t edq_lost_packed(const EdqAcc& a) { return (a.lost & 0xFFFFu) + (a.lost >> 16); }

@@ -85,3 +85,21 @@ def edq_close(got: dict, want: dict, rel=1e-5):
         a, b = got[k], want[k]
         assert abs(a - b) <= rel * abs(b) + 1e-300, (k, a, b)
     assert got["lost"] == want["lost"], ("lost", got["lost"], want["lost"])
+
+
+def resplit_pairs(update_bits: int):
+    """Normalised pairs (x, y) on which Grow((x, y), update) returns the same value x + y split over other
+    components: the parameter has not moved although both stored patterns changed.  Input selection only
+    (expected results always come from the oracle's step); found by scanning windows with the oracle's Grow."""
+    hi = np.concatenate([np.arange(0x3E80, 0x4080), np.arange(0xBE80, 0xC080)]).astype(np.uint16)
+    lo = np.concatenate([np.arange(0x3900, 0x3C01), np.arange(0xB900, 0xBC01)]).astype(np.uint16)
+    x, y = np.repeat(hi, lo.size), np.tile(lo, hi.size)
+    f = lambda b: (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    ulp = np.ldexp(1.0, (((x >> 7) & 0xFF).astype(np.int32) - 127 - 7))
+    ok = np.abs(f(y)) <= ulp / 2
+    x, y = x[ok], y[ok]
+    u, v = oracle.grow(x, y, np.full(x.size, update_bits, np.uint16))
+    same_value = f(u) + f(v) == f(x) + f(y)            # exact in double: all terms within a few binades
+    moved_bits = (f(u) != f(x)) | (f(v) != f(y))
+    pick = same_value & moved_bits
+    return x[pick], y[pick]

@@ -164,6 +164,13 @@ def test_standalone_edq_matches_oracle():
     delta = rng.choice(bf16_window(-16, -9, with_zero=True), n)
     new_hi, new_lo = oracle.grow(old_hi, old_lo, delta)
     new_hi[::7] = old_hi[::7]; new_lo[::7] = old_lo[::7]            # some lost updates
+    # and some where Grow re-splits the same value over other components: not updated either (value reading)
+    from gpu_util import resplit_pairs
+    xs, ys = resplit_pairs(0x35AB)
+    kp = np.arange(3, n, 13)
+    old_hi[kp], old_lo[kp], delta[kp] = xs[kp % xs.size], ys[kp % xs.size], 0x35AB
+    new_hi[kp], new_lo[kp] = oracle.grow(old_hi[kp], old_lo[kp], delta[kp])
+    assert np.all((new_hi[kp] != old_hi[kp]) | (new_lo[kp] != old_lo[kp]))
     dev = [Guarded(a, 1) for a in (old_hi, old_lo, new_hi, new_lo, delta)]
     out = torch.zeros(64, dtype=torch.uint8, device="cuda")
     ws = torch.empty(B.workspace_bytes(), dtype=torch.uint8, device="cuda")
@@ -178,6 +185,8 @@ def test_standalone_edq_matches_oracle():
         for k in ("dot", "sumsq", "edq"):
             assert abs(got[k] - want[k]) <= 1e-5 * abs(want[k])
         assert got["lost"] == want["lost"] and got["n"] == n
+        if has_lo:
+            assert got["lost"] >= kp.size + n // 7 - kp.size // 7 - 2
 
 
 def test_standalone_edq_past_2_to_32_elements_is_the_sum_of_its_pieces():

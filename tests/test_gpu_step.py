@@ -144,7 +144,10 @@ def test_stress_lost_arithmetic_config_short():
             hist.append(got)
         _compare(dev, st, f"stress strategy {strategy}")
         edq_hist[strategy] = hist
-    # plain bfloat16 loses most updates here, Collage-plus only the few below the reach of its second component
+    # plain bfloat16 loses most updates here (Def. 3.2: |update| <= ulp(theta)/2).  Collage-plus loses only those
+    # below the reach of its second component: a length-2 bfloat16 expansion resolves about 2^-17 |theta|
+    # (|dtheta| <= ulp(theta)/2 = 2^-9 |theta|, and dtheta has 8 bits of its own), and with lr 1e-5 and gradients
+    # down to 1e-8 a few per cent of the updates are smaller than that; hence 5 %, not 0
     assert edq_hist[0][-1]["lost"] > 0.5 * n
     assert edq_hist[2][-1]["lost"] < 0.05 * n
     assert edq_hist[2][-1]["edq"] > edq_hist[0][-1]["edq"]
@@ -364,3 +367,41 @@ def test_hyper_parameter_and_step_sweep(strategy):
         want = oracle_step(st, g, t, strategy, hyp)
         _compare(dev, st, f"hypers {hyp} step {t} strategy {strategy}")
         edq_close(e.read(), want)
+
+
+@pytest.mark.parametrize("strategy", [1, 2])
+def test_lost_counts_values_that_did_not_move_on_planted_resplit_pairs(strategy):
+    # Pairs on which Grow hands back the same value over other components, planted densely: the count
+    # follows the value (Eq. 2's effective update is zero), not the stored bit patterns.  beta1 = beta2 = 0,
+    # no decay and g = -+1 make the update exactly +-RN(lr) at step 1, so the planted update is what the step applies.
+    from gpu_util import resplit_pairs
+    a_bits = 0x35AB
+    lr = float(oracle.widen(a_bits))
+    hyp = dict(lr=lr, beta1=0.0, beta2=0.0, eps=1e-8, weight_decay=0.0)
+    xp, yp = resplit_pairs(a_bits)                       # update +a
+    xm, ym = resplit_pairs(a_bits | 0x8000)              # update -a
+    assert xp.size > 500 and xm.size > 500
+    rng = np.random.default_rng(99)
+    n = 300_011
+    th = W.bits(W.stress_weights(n, 5)); dth = np.zeros(n, np.uint16)
+    g = np.where(rng.integers(0, 2, n) == 1, np.uint16(0x3F80), np.uint16(0xBF80)).astype(np.uint16)
+    planted = rng.random(n) < 0.5
+    for sign_bits, (xs, ys) in ((0xBF80, (xp, yp)), (0x3F80, (xm, ym))):      # g = -1 gives +a, g = +1 gives -a
+        idx = np.flatnonzero(planted & (g == sign_bits))
+        k = rng.integers(0, xs.size, idx.size)
+        th[idx], dth[idx] = xs[k], ys[k]
+    st = oracle_state(th, strategy)
+    st["x_lo"] = dth.copy()
+    before = (st["x_hi"].copy(), st["x_lo"].copy())
+    dev = _device_state(st)
+    e = EdqBuffers()
+    G = Guarded(g)
+    B.adamw_step(_t(dev["x_hi"]), _t(dev["x_lo"]), _t(dev["m"]), _t(dev["v_hi"]), _t(dev["v_lo"]), G.t, n, e.hyper(hyp), 1, strategy)
+    torch.cuda.synchronize()
+    want = oracle_step(st, g, 1, strategy, hyp)
+    _compare(dev, st, f"planted resplit pairs, strategy {strategy}")
+    got = e.read()
+    edq_close(got, want)
+    components_same = int(np.sum((st["x_hi"] == before[0]) & (st["x_lo"] == before[1])))
+    assert got["lost"] >= int(planted.sum()) > n // 3            # every planted pair is counted ...
+    assert got["lost"] - components_same >= int(planted.sum())   # ... and none of them kept its bit patterns
