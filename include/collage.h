@@ -28,7 +28,14 @@
  *   - pointers need not be 16-byte aligned and lengths need not be multiples of 8 (such
  *     tensors take a slower element-wise path with identical results);
  *   - n == 0 is a successful no-op;
- *   - NaN/Inf in tensor data is not an error: it propagates per IEEE 754.
+ *   - NaN/Inf in tensor data is not an error: it propagates per IEEE 754;
+ *   - threads: any entry point may be called from several host threads at once, on the same or on
+ *     different devices and streams (the library's own first-call set-up is guarded), provided that
+ *     calls in flight together share no tensor, no workspace, no plan being modified
+ *     (collage_plan_set_replicas, collage_plan_destroy) and, for collage_adamw_step_host and
+ *     collage_edq_static, no device: those two keep one context or scratch array per device;
+ *   - the EDQ workspace (hyper->workspace) must hold zeros before its first use: clear it once with
+ *     collage_workspace_init or cudaMemset.  Every call leaves it ready for the next one.
  */
 #ifndef COLLAGE_H_
 #define COLLAGE_H_
@@ -44,7 +51,7 @@ typedef enum {
     COLLAGE_OK = 0,
     COLLAGE_ERR_NULL = 1,       /* a required pointer is NULL                                   */
     COLLAGE_ERR_ARG = 2,        /* step == 0, unknown strategy/op/flag combination, hyper out of range */
-    COLLAGE_ERR_ALIAS = 3,      /* two tensors of one call overlap                              */
+    COLLAGE_ERR_ALIAS = 3,      /* two tensors of one call overlap, or one overlaps the workspace / EDQ record */
     COLLAGE_ERR_ARCH = 4,       /* current device is not sm_100                                 */
     COLLAGE_ERR_CUDA = 5,       /* a CUDA runtime call or launch failed                         */
     COLLAGE_ERR_WORKSPACE = 6,  /* workspace missing or smaller than collage_workspace_bytes()  */
@@ -96,12 +103,15 @@ typedef struct collage_hyper {
  *   lost  = #{i : delta_i != 0 and eff_i == 0}: parameters that an update was meant for and that did not
  *           move (Def. 3.2; "not updated", Figure 3 left).  For a pair the value theta + dtheta counts:
  *           a Grow that re-splits the same value over other components has not updated it.
+ *   fault = 0, or the code of a bounded device-side wait that gave up during this call (see
+ *           collage_pipeline_fault): the step was torn and the state arrays are then undefined.
  * Products and 8-element partial sums are formed in float, everything above in double, in a
  * fixed order: the result is reproducible for a given launch geometry. */
 typedef struct collage_edq {
     double dot, sumsq, edq;
     uint64_t n;
     uint64_t lost;
+    uint64_t fault;
 } collage_edq_t;
 
 /* One parameter tensor of a multi-tensor plan.  x_lo may be NULL for a plan used only with
@@ -129,16 +139,38 @@ const char* collage_status_string(collage_status_t status);
  * Errors: NULL -> ERR_NULL; step == 0 or hyper out of range -> ERR_ARG. */
 collage_status_t collage_derive_scalars(const collage_hyper_t* hyper, uint64_t step, uint16_t out_bf16[11]);
 
-/* Bytes of device scratch the EDQ reduction needs (independent of n; a few tens of KiB). */
+/* Bytes of device scratch the EDQ reduction needs (independent of n; about 128 KiB). */
 size_t collage_workspace_bytes(uint64_t n_total);
+
+/* Clears an EDQ workspace (asynchronous memset on `stream`).  The step kernels end their EDQ
+ * reduction (Eq. 3) inside the same launch: each thread block stores its partial sums in the
+ * workspace and draws a ticket from a counter that lives there; the block that draws the last
+ * ticket adds the partials in index order and writes the record.  The counter wraps back to zero
+ * with the last ticket, so one clearing before the first use is enough.  A workspace serves one
+ * call at a time: calls that may run concurrently need separate workspaces.
+ * Errors: ERR_NULL, ERR_WORKSPACE (smaller than collage_workspace_bytes() or not 16-byte aligned),
+ * ERR_CUDA. */
+collage_status_t collage_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Combines EDQ records of disjoint parameter sets (tensors, slices, ranks) into the record of their
+ * union, Eq. 3 on the summed partial sums: dot, sumsq, n and lost are added in array order, edq =
+ * dot / sqrt(sumsq) (0 if sumsq == 0), fault = the first non-zero fault.  HOST arrays, no CUDA call.
+ * `out` may be one of the parts.  Errors: ERR_NULL, ERR_ARG (count < 0). */
+collage_status_t collage_edq_combine(const collage_edq_t* parts_host, int count, collage_edq_t* out_host);
+
+/* "product" for the ordinary build; a measurement build of the same sources that compiles the
+ * arithmetic out of the step kernel (to time the copy pipeline alone) answers "data-movement-only". */
+const char* collage_build_flavor(void);
 
 /* One AdamW step over one flat tensor (Algorithm 2 lines 8-13, all n parameters, step t >= 1).
  *   x_hi, m, v_hi, grad : required.   x_lo : required iff strategy != COLLAGE_BF16 (delta-theta, or
  *   the Kahan compensation for COLLAGE_KAHAN), else must
  *   be NULL.   v_lo : required iff strategy is COLLAGE_PLUS or COLLAGE_PLUS_FP32_REGISTERS, else
  *   must be NULL.
+ * With hyper->edq_out set the record is written by the same launch (one kernel per step).
  * Errors: ERR_NULL, ERR_ARG (step 0, bad strategy, hyper range), ERR_ALIAS (overlapping
- * tensors), ERR_WORKSPACE (edq_out set, workspace too small), ERR_ARCH, ERR_CUDA. */
+ * tensors; workspace or record overlapping a tensor or each other), ERR_WORKSPACE (edq_out set,
+ * workspace missing, misaligned or too small), ERR_ARCH, ERR_CUDA. */
 collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi, void* v_lo,
                                     const void* grad, uint64_t n, const collage_hyper_t* hyper,
                                     uint64_t step, collage_strategy_t strategy, void* stream);
@@ -209,10 +241,17 @@ collage_status_t collage_plan_destroy(collage_plan_t* plan);
  *              0 removes the replicas.
  * The call synchronises the device and allocates a small table: do it once, outside the step loop.
  * A replica holds the new theta once the step's kernel has finished; readers on other GPUs need
- * their own ordering with that (an event, a barrier).  Plain bulk stores only, no multicast.
+ * their own ordering with that (an event, a barrier).  Plain stores issued by each block for itself.
  * Errors: ERR_NULL, ERR_ARG (count, alignment, wrong device), ERR_ALIAS (a replica overlaps an
  * array of the plan or another replica), ERR_CUDA. */
 collage_status_t collage_plan_set_replicas(collage_plan_t* plan, const void* const* replicas, int num_replicas);
+
+/* Lets kernels of the CURRENT device store into memory of `peer_device` (a device ordinal of this
+ * process), so that pointers into a peer's memory that the caller has mapped (CUDA IPC, virtual
+ * memory management) can serve as replicas.  Host-side set-up, not on the step path; succeeds if the
+ * access is already enabled.  The paper has no counterpart (its experiments do not shard the step).
+ * Errors: ERR_ARG (same device, or the devices cannot reach each other), ERR_CUDA. */
+collage_status_t collage_enable_peer_access(int peer_device);
 
 /* The multi-tensor step with EDQ kept per tensor (Eq. 2-3 evaluated on each parameter tensor of the
  * plan separately; the lost-update count of Def. 3.2 per tensor gives the imprecision percentage of
@@ -224,7 +263,7 @@ collage_status_t collage_plan_set_replicas(collage_plan_t* plan, const void* con
  *   hyper->edq_out     : optional DEVICE collage_edq_t for the whole plan = the per-tensor sums added
  *                        in tensor order (association differs from collage_adamw_step_multi's, so
  *                        the last bits may differ); hyper->workspace is not used by this call.
- * Three launches (step, per-tensor sums, total) instead of two.  The variant flags (TWOSUM_GROW,
+ * Three launches (step, per-tensor sums, total) instead of one.  The variant flags (TWOSUM_GROW,
  * DECAY_BY_GROW) are not available through this entry point (ERR_ARG).
  * Errors: as collage_adamw_step_multi, plus ERR_ARG when num differs from the plan's and
  * ERR_WORKSPACE for the chunk workspace. */
@@ -278,8 +317,8 @@ collage_status_t collage_edq(const void* old_hi, const void* old_lo, const void*
  * into the library: a fixed 64 KiB array in device memory (2048 partial sums), which every GPU
  * that loads the library holds until the process exits.  Arguments are those of collage_edq
  * without workspace; `out_dev` is still the caller's DEVICE collage_edq_t.
- *   - Capacity: one partial sum per 2^21 elements, so n <= 2^32; a larger n is rejected with
- *     COLLAGE_ERR_LIMIT and nothing is launched.
+ *   - Capacity: the array has 2048 slots and a thread block reduces up to 2^21 elements, so
+ *     n <= 2^32; a larger n is rejected with COLLAGE_ERR_LIMIT and nothing is launched.
  *   - The call itself allocates nothing and frees nothing.  The first call on each device looks up
  *     the array's device address (cudaGetSymbolAddress, with that device current); make that first
  *     call before any stream capture begins.
@@ -287,23 +326,27 @@ collage_status_t collage_edq(const void* old_hi, const void* old_lo, const void*
  *     so nothing needs clearing between calls; but two calls whose kernels overlap on the GPU
  *     (different streams, no ordering) race on it.  Order them, or use collage_edq with separate
  *     workspaces.
- *   - The sums are grouped per fixed 2^21-element segment, not per launch geometry, so they can
- *     differ from collage_edq's in the last bits (same tolerance as against the CPU oracle).
+ *   - The sums are grouped per segment of ceil(n / 2048) elements (rounded up to a multiple of 8,
+ *     at least 2048), a function of n alone and not of the launch geometry, so they can differ from
+ *     collage_edq's in the last bits (same tolerance as against the CPU oracle).
  * Errors: ERR_NULL, ERR_LIMIT, ERR_ARCH, ERR_CUDA. */
 collage_status_t collage_edq_static(const void* old_hi, const void* old_lo, const void* new_hi,
                                     const void* new_lo, const void* delta, uint64_t n,
                                     collage_edq_t* out_dev, void* stream);
 
-/* The step kernel's copy pipeline waits on shared-memory barriers with a bound of about two
- * seconds; a wait that runs out records a code in a device word and the block leaves, so a fault
- * can never hang the device.  This call copies that word to *out_host (0 = no fault ever seen on
- * the current device since the last read) and clears it.  It synchronises the device: call it at
- * checkpoints, not per step.  Errors: ERR_NULL, ERR_CUDA. */
+/* The step kernel's copy pipeline waits on shared-memory barriers with a bound of two seconds of
+ * the device's wall clock; a wait that runs out records a code in a device word and the block
+ * leaves, so a fault can never hang the device.  The kernel still ends normally and the call has
+ * long returned COLLAGE_OK, but the step was torn: the state arrays are undefined from then on.
+ * A step that reduces EDQ copies the word into its record (collage_edq_t.fault), so a caller that
+ * reads the record sees the fault at once.  This call copies the word to *out_host (0 = no fault
+ * seen on the current device since the last read) and clears it.  It synchronises the device: call
+ * it at checkpoints, not per step.  Errors: ERR_NULL, ERR_CUDA. */
 collage_status_t collage_pipeline_fault(uint32_t* out_host);
 
 /* Exercises the give-up path of those waits without any fault: launches one warp that waits on a
- * barrier nothing completes, bounded by about `limit_ms` milliseconds (1..1000, counted in SM
- * cycles at 2 GHz).  The wait runs out, the kernel returns normally, and the next
+ * barrier nothing completes, bounded by `limit_ms` milliseconds (1..1000) of the device's wall
+ * clock.  The wait runs out, the kernel returns normally, and the next
  * collage_pipeline_fault reports the code 100.  The device and the library stay usable.
  * Asynchronous on `stream`.  Errors: ERR_ARG (limit out of range), ERR_ARCH, ERR_CUDA. */
 collage_status_t collage_wait_timeout_selftest(uint32_t limit_ms, void* stream);

@@ -7,12 +7,9 @@ There is no fallback: if the shared library has not been built, loading raises.
 from __future__ import annotations
 
 import ctypes
-import os
 from pathlib import Path
 
-# the in-tree build, unless COLLAGE_B200_LIB names another build of the same sources (see build.py --out)
-_LIB_PATH = Path(os.environ["COLLAGE_B200_LIB"]).resolve() if os.environ.get("COLLAGE_B200_LIB") \
-    else Path(__file__).resolve().parent / "libcollage_b200.so"
+_LIB_PATH = Path(__file__).resolve().parent / "libcollage_b200.so"      # the in-tree build
 
 OK, ERR_NULL, ERR_ARG, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_WORKSPACE, ERR_LIMIT = range(8)
 BF16, LIGHT, PLUS, KAHAN, PLUS_FP32_REGISTERS = 0, 1, 2, 3, 4
@@ -28,6 +25,7 @@ EXPORTS = (
     "collage_fast_two_sum", "collage_two_sum", "collage_two_prod", "collage_grow",
     "collage_scaling", "collage_mul", "collage_renormalize", "collage_rounded_op", "collage_edq",
     "collage_selftest", "collage_pipeline_fault", "collage_edq_static", "collage_wait_timeout_selftest",
+    "collage_workspace_init", "collage_edq_combine", "collage_build_flavor", "collage_enable_peer_access",
 )
 
 
@@ -41,7 +39,10 @@ class Hyper(ctypes.Structure):
 class Edq(ctypes.Structure):
     """collage_edq_t"""
     _fields_ = [("dot", ctypes.c_double), ("sumsq", ctypes.c_double), ("edq", ctypes.c_double),
-                ("n", ctypes.c_uint64), ("lost", ctypes.c_uint64)]
+                ("n", ctypes.c_uint64), ("lost", ctypes.c_uint64), ("fault", ctypes.c_uint64)]
+
+
+EDQ_RECORD_BYTES = ctypes.sizeof(Edq)
 
 
 class Tensor(ctypes.Structure):
@@ -58,16 +59,30 @@ class CollageError(RuntimeError):
 
 
 _lib = None
+_lib_path = _LIB_PATH
+
+
+def load(path) -> ctypes.CDLL:
+    """Use another build of the same sources (``build.py --out``) instead of the in-tree library.
+
+    Only an explicit call selects it (the benchmark's ``--lib``); nothing in the environment can swap
+    the library under a caller.  Must come before the first use of the library in this process.
+    """
+    global _lib_path
+    if _lib is not None:
+        raise RuntimeError("the library is already loaded; call load() before any other function")
+    _lib_path = Path(path).resolve()
+    return lib()
 
 
 def lib() -> ctypes.CDLL:
     """The loaded CUDA library; raises if it has not been built (there is no other path)."""
     global _lib
     if _lib is None:
-        if not _LIB_PATH.exists():
-            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2405_03637_b200.build` "
+        if not _lib_path.exists():
+            raise RuntimeError(f"{_lib_path} is missing: build it with `python -m paper_2405_03637_b200.build` "
                                "(this package has no CPU or PyTorch fallback)")
-        L = ctypes.CDLL(str(_LIB_PATH))
+        L = ctypes.CDLL(str(_lib_path))
         vp, u64, i32 = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_int
         L.collage_status_string.restype = ctypes.c_char_p
         L.collage_status_string.argtypes = [i32]
@@ -101,6 +116,11 @@ def lib() -> ctypes.CDLL:
         L.collage_selftest.argtypes = [ctypes.POINTER(ctypes.c_uint64), vp]
         L.collage_pipeline_fault.argtypes = [ctypes.POINTER(ctypes.c_uint32)]
         L.collage_wait_timeout_selftest.argtypes = [ctypes.c_uint32, ctypes.c_void_p]
+        L.collage_workspace_init.argtypes = [vp, ctypes.c_size_t, vp]
+        L.collage_edq_combine.argtypes = [ctypes.POINTER(Edq), i32, ctypes.POINTER(Edq)]
+        L.collage_build_flavor.restype = ctypes.c_char_p
+        L.collage_build_flavor.argtypes = []
+        L.collage_enable_peer_access.argtypes = [i32]
         _lib = L
     return _lib
 
@@ -137,6 +157,30 @@ def derive_scalars(hyper: Hyper, step: int) -> dict:
 
 def workspace_bytes(n_total: int = 0) -> int:
     return int(lib().collage_workspace_bytes(n_total))
+
+
+def workspace_init(workspace, stream=None):
+    """Clear an EDQ workspace (a CUDA uint8 tensor): needed once, before its first use."""
+    _check(lib().collage_workspace_init(_ptr(workspace), workspace.numel() * workspace.element_size(), _ptr(stream)),
+           "collage_workspace_init")
+
+
+def _record(rec: Edq) -> dict:
+    return dict(dot=rec.dot, sumsq=rec.sumsq, edq=rec.edq, n=int(rec.n), lost=int(rec.lost), fault=int(rec.fault))
+
+
+def edq_combine(parts) -> dict:
+    """EDQ record of the union of disjoint parameter sets from their records (dicts with dot, sumsq, n, lost)."""
+    arr = (Edq * max(len(parts), 1))()
+    for i, p in enumerate(parts):
+        arr[i] = Edq(p["dot"], p["sumsq"], p.get("edq", 0.0), p.get("n", 0), p["lost"], p.get("fault", 0))
+    out = Edq()
+    _check(lib().collage_edq_combine(arr, len(parts), ctypes.byref(out)), "collage_edq_combine")
+    return _record(out)
+
+
+def build_flavor() -> str:
+    return lib().collage_build_flavor().decode()
 
 
 def adamw_step(x_hi, x_lo, m, v_hi, v_lo, grad, n, hyper: Hyper, step: int, strategy: int, stream=None):
@@ -180,13 +224,18 @@ def plan_set_replicas(plan: int, replicas):
     _check(lib().collage_plan_set_replicas(plan, arr, len(replicas)), "collage_plan_set_replicas")
 
 
+def enable_peer_access(peer_device: int):
+    """Let kernels of the current device store into `peer_device`'s memory (set-up for replicas on other GPUs)."""
+    _check(lib().collage_enable_peer_access(peer_device), "collage_enable_peer_access")
+
+
 def plan_workspace_bytes(plan: int) -> int:
     return int(lib().collage_plan_workspace_bytes(plan))
 
 
 def adamw_step_multi_per_tensor(plan: int, hyper: Hyper, step: int, strategy: int, per_tensor_out, num: int,
                                 chunk_workspace, stream=None):
-    """per_tensor_out: CUDA uint8 tensor of num * 40 bytes; chunk_workspace: CUDA uint8 tensor."""
+    """per_tensor_out: CUDA uint8 tensor of num * EDQ_RECORD_BYTES bytes; chunk_workspace: CUDA uint8 tensor."""
     _check(lib().collage_adamw_step_multi_per_tensor(plan, ctypes.byref(hyper), step, strategy, _ptr(per_tensor_out), num,
                                                      _ptr(chunk_workspace),
                                                      chunk_workspace.numel() * chunk_workspace.element_size(),
@@ -198,8 +247,7 @@ def read_edq_array(dev_bytes, num: int) -> list:
     raw = dev_bytes.detach().cpu().numpy().tobytes()
     out = []
     for i in range(num):
-        rec = Edq.from_buffer_copy(raw[i * ctypes.sizeof(Edq):(i + 1) * ctypes.sizeof(Edq)])
-        out.append(dict(dot=rec.dot, sumsq=rec.sumsq, edq=rec.edq, n=int(rec.n), lost=int(rec.lost)))
+        out.append(_record(Edq.from_buffer_copy(raw[i * ctypes.sizeof(Edq):(i + 1) * ctypes.sizeof(Edq)])))
     return out
 
 
@@ -277,7 +325,6 @@ def wait_timeout_selftest(limit_ms: int, stream=None):
 
 
 def read_edq(edq_dev) -> dict:
-    """Copy a device collage_edq_t (a >= 40-byte torch.uint8 CUDA tensor) to the host and decode it."""
+    """Copy a device collage_edq_t (a >= EDQ_RECORD_BYTES torch.uint8 CUDA tensor) to the host and decode it."""
     raw = edq_dev.detach().cpu().numpy().tobytes()
-    rec = Edq.from_buffer_copy(raw[:ctypes.sizeof(Edq)])
-    return dict(dot=rec.dot, sumsq=rec.sumsq, edq=rec.edq, n=int(rec.n), lost=int(rec.lost))
+    return _record(Edq.from_buffer_copy(raw[:ctypes.sizeof(Edq)]))

@@ -5,7 +5,7 @@
 --define adds a preprocessor definition (the geometry constants COLLAGE_PIPE_* / COLLAGE_FP32_*, or
 COLLAGE_DATA_MOVEMENT_ONLY, which compiles the arithmetic out of the step kernel to measure what the
 copy pipeline alone sustains); such a build goes to --out, never over the in-tree library, and is
-loaded by pointing the environment variable COLLAGE_B200_LIB at it.
+loaded only on request: `binding.load(path)`, which `bench.py --lib PATH` calls.
 
 The exactness of the error-free transforms depends on the flags below: no FMA contraction,
 no flush-to-zero, IEEE division and square root, never --use_fast_math.

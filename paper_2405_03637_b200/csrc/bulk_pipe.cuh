@@ -1,6 +1,6 @@
 // Building blocks of the bulk-copy pipelines: shared-memory mbarriers with bounded waits and the
-// 1-D bulk asynchronous copies (cp.async.bulk) between global and shared memory.  No multicast
-// form is used anywhere.
+// 1-D bulk asynchronous copies between global and shared memory, each issued by one block for
+// itself (plain per-block copies only).
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -31,18 +31,24 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after `limit` cycles (by default ~4e9, about two seconds) and records in
+// nanoseconds of the device's wall clock (independent of the SM clock)
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after `limit_ns` nanoseconds (two seconds by default) and records in
 // *fault_word which wait failed (1 + who; the first failure wins).  The caller leaves its loops
 // when this returns false.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int who, unsigned int* fault_word,
-                                          long long limit = 4000000000LL) {
+                                          unsigned long long limit_ns = 2000000000ULL) {
     if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
+    const unsigned long long t0 = global_ns();
     for (;;) {
 #pragma unroll 1
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > limit) {
+        if (global_ns() - t0 > limit_ns) {
             atomicCAS(fault_word, 0u, who + 1u);
             return false;
         }

@@ -13,9 +13,18 @@ void launch_edq_finalize(const EdqPartial* partials, int count, uint64_t n, coll
                          bool accumulate);
 
 constexpr int kStaticThreads = 256;
-constexpr uint64_t kSegment = 1ull << 21;                    // elements reduced by one block
 constexpr int kStaticPartials = 2048;                        // 2048 x 32 B = 64 KiB of scratch
-constexpr uint64_t kStaticMaxN = kSegment * kStaticPartials; // 2^32 elements
+constexpr uint64_t kStaticMaxN = 1ull << 32;                 // elements; one block then reduces 2^21 of them
+constexpr uint64_t kMinSegment = 2048;                       // elements reduced by one block, at least
+
+// Elements per block for a tensor of n elements: enough blocks to fill the GPU at every size, never
+// more than the scratch has slots, a whole number of 8-element vectors.  A function of n alone, so
+// the grouping of the sums, and with it the result, is the same on every device.
+inline uint64_t static_segment(uint64_t n) {
+    uint64_t seg = (n + kStaticPartials - 1) / kStaticPartials;
+    seg = (seg + 7) & ~7ull;
+    return seg < kMinSegment ? kMinSegment : seg;
+}
 
 // The scratch itself.  In host code this name is only a handle for cudaGetSymbolAddress; it is
 // not a device address and must never be passed to a kernel as one.
@@ -28,16 +37,17 @@ struct StaticEdqArgs {
     const uint16_t* new_lo;
     const uint16_t* delta;
     uint64_t n;
+    uint64_t segment;         // elements per block
     int aligned;
     EdqPartial* partials;     // device address of g_static_partials, looked up by the host
 };
 
-// Block b reduces elements [b * kSegment, (b+1) * kSegment) and overwrites partial b: every slot
+// Block b reduces elements [b * segment, (b+1) * segment) and overwrites partial b: every slot
 // that the finalize kernel will read is written by this launch, so stale contents never matter.
 template <bool HAS_LO>
 __global__ void __launch_bounds__(kStaticThreads) edq_static_kernel(const __grid_constant__ StaticEdqArgs p) {
-    const uint64_t seg_begin = blockIdx.x * kSegment;
-    const uint64_t seg_end = (p.n - seg_begin < kSegment) ? p.n : seg_begin + kSegment;
+    const uint64_t seg_begin = blockIdx.x * p.segment;
+    const uint64_t seg_end = (p.n - seg_begin < p.segment) ? p.n : seg_begin + p.segment;
     const uint64_t nvec = (seg_end - seg_begin + 7) >> 3;
     double dot = 0.0, sq = 0.0;
     unsigned long long lost = 0;
@@ -95,20 +105,21 @@ __global__ void __launch_bounds__(kStaticThreads) edq_static_kernel(const __grid
     }
 }
 
-// Device address of the static scratch on the current device, looked up once per device.
+// Device address of the static scratch on the current device, looked up once per device.  Host
+// threads racing on the first call look the same address up twice and store it twice.
 static cudaError_t static_scratch(EdqPartial** out) {
-    static EdqPartial* address[64] = {};
+    static std::atomic<EdqPartial*> address[64];
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
-    if (!address[dev]) {
-        EdqPartial* ptr = nullptr;
+    EdqPartial* ptr = address[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_partials);   // `dev` is current
         if (e != cudaSuccess) return e;
-        address[dev] = ptr;
+        address[dev].store(ptr, std::memory_order_release);
     }
-    *out = address[dev];
+    *out = ptr;
     return cudaSuccess;
 }
 
@@ -138,7 +149,8 @@ extern "C" collage_status_t collage_edq_static(const void* old_hi, const void* o
                            reinterpret_cast<uintptr_t>(delta);
     p.aligned = (bits & 15u) == 0;
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
-    const unsigned grid = static_cast<unsigned>((n + kSegment - 1) / kSegment);
+    p.segment = static_segment(n);
+    const unsigned grid = static_cast<unsigned>((n + p.segment - 1) / p.segment);
     if (grid > 0) {
         if (old_lo) edq_static_kernel<true><<<grid, kStaticThreads, 0, cs>>>(p);
         else edq_static_kernel<false><<<grid, kStaticThreads, 0, cs>>>(p);

@@ -9,6 +9,7 @@
 // m 4, v 4, w 4), D^-MW 22 B.
 #include "bulk_pipe.cuh"
 #include "host_common.cuh"
+#include "edq_reduce.cuh"
 #include "mcf_device.cuh"
 
 namespace collage {
@@ -34,7 +35,7 @@ struct Fp32Params {
     uint64_t n;
     int aligned;          // every pointer is 16-byte aligned
     Fp32Scalars k;
-    EdqPartial* partials;
+    EdqFinish fin;              // per-block partials, ticket and record of the EDQ reduction
 };
 
 // Geometry of the pipeline (one block per SM, a producer warp beside the consumers).  The version
@@ -79,6 +80,7 @@ struct Fp32Smem {
     alignas(8) uint64_t done[kStages];
     double red_dot[kCons / 32], red_sq[kCons / 32];
     unsigned long long red_lost[kCons / 32];
+    EdqFinishSmem finish;
 };
 
 // One parameter: Algorithm 2 lines 8-13 in float.  Returns the update; w is the stored float
@@ -284,17 +286,18 @@ __global__ void __launch_bounds__(Fp32Geometry<MASTER>::kCons + 32, 1) adamw_fp3
             }
         }
         __syncthreads();
+        double d = 0.0, q = 0.0;
+        unsigned long long l = 0;
         if (threadIdx.x == 0) {
-            double d = 0.0, q = 0.0;
-            unsigned long long l = 0;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) {
                 d += sm.red_dot[w];
                 q += sm.red_sq[w];
                 l += sm.red_lost[w];
             }
-            p.partials[blockIdx.x] = EdqPartial{d, q, l, 0ull};
         }
+        // one partial per block; the block that finishes last adds them up and writes the record
+        edq_publish_and_finish(p.fin, sm.finish, d, q, l, &g_pipeline_fault32);
     }
 }
 
@@ -303,13 +306,13 @@ static cudaError_t launch_fp32(const Fp32Params& p, int sm_count, cudaStream_t s
     auto kernel = adamw_fp32_pipeline_kernel<MASTER, EDQ>;
     constexpr size_t smem = sizeof(Fp32Smem<MASTER>) + 128;
     constexpr int kTile32 = Fp32Geometry<MASTER>::kTile, kCons32 = Fp32Geometry<MASTER>::kCons;
-    static bool ready[64] = {};
+    static std::atomic<bool> ready[64];     // racing first calls set the same attribute twice: harmless
     int device = 0;
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return cudaErrorInvalidDevice;
-    if (!ready[device]) {
+    if (!ready[device].load(std::memory_order_acquire)) {
         const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
-        ready[device] = true;
+        ready[device].store(true, std::memory_order_release);
     }
     const uint64_t tiles = (p.n + kTile32 - 1) / kTile32;
     uint64_t grid = static_cast<uint64_t>(sm_count);
@@ -342,6 +345,7 @@ extern "C" collage_status_t collage_adamw_step_fp32(void* theta, void* master, v
         if (!hyper->workspace || hyper->workspace_bytes < kWorkspaceBytes ||
             (reinterpret_cast<uintptr_t>(hyper->workspace) & 15u))
             return COLLAGE_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(hyper->edq_out) & 7u) return COLLAGE_ERR_ARG;
     }
     if (!theta || !m || !v || !grad) return COLLAGE_ERR_NULL;
     if (n > (1ull << 61)) return COLLAGE_ERR_ARG;
@@ -356,6 +360,10 @@ extern "C" collage_status_t collage_adamw_step_fp32(void* theta, void* master, v
     add(m, 4 * n);
     add(v, 4 * n);
     add(master, 4 * n);
+    if (hyper->edq_out) {
+        add(hyper->edq_out, sizeof(collage_edq_t));
+        add(hyper->workspace, kWorkspaceBytes);
+    }
     if (any_overlap(ranges)) return COLLAGE_ERR_ALIAS;
     DeviceInfo dev;
     const collage_status_t st = current_device(&dev);
@@ -381,7 +389,13 @@ extern "C" collage_status_t collage_adamw_step_fp32(void* theta, void* master, v
     p.k.lam = static_cast<float>(hyper->weight_decay);
     p.k.eps = static_cast<float>(hyper->eps);
     p.k.flags = hyper->flags;
-    p.partials = static_cast<EdqPartial*>(hyper->workspace);
+    if (hyper->edq_out) {
+        p.fin.partials = static_cast<EdqPartial*>(hyper->workspace);
+        p.fin.ticket = reinterpret_cast<unsigned int*>(static_cast<char*>(hyper->workspace) + kTicketOffset);
+        p.fin.out = static_cast<collage_edq_t*>(hyper->edq_out);
+        p.fin.n = n;
+        p.fin.accumulate = 0;
+    }
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     const bool edq = hyper->edq_out != nullptr;
     int grid = 0;
@@ -391,8 +405,8 @@ extern "C" collage_status_t collage_adamw_step_fp32(void* theta, void* master, v
         else e = edq ? launch_fp32<false, true>(p, dev.sm_count, cs, &grid) : launch_fp32<false, false>(p, dev.sm_count, cs, &grid);
         if (e != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
-    if (edq) {
-        launch_edq_finalize(p.partials, grid, n, static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
+    if (edq && grid == 0) {        // nothing was launched (n == 0): the record still has to say so
+        launch_edq_finalize(p.fin.partials, 0, 0, p.fin.out, cs, false);
         if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
     return COLLAGE_OK;

@@ -7,9 +7,12 @@
 // shared memory, 8 consecutive elements (one 16-byte vector per state array) at a time.  Tensors
 // whose pointers are not all 16-byte aligned, and the ragged end of a tensor, go through plain or
 // element-wise accesses that feed the same arithmetic.  EDQ sums: float within a vector, double
-// per thread, fixed-order tree per block, one partial per block, summed by a one-block finalize
-// kernel.
+// per thread, fixed-order tree per block, one partial per block, summed by the block that
+// finishes last (edq_reduce.cuh): a step is one launch.
+#include <mutex>
+
 #include "host_common.cuh"
+#include "edq_reduce.cuh"
 #include "mcf_device.cuh"
 
 // Geometry of the pipeline kernel.  Measured on B200 (2^30 parameters, Collage-plus with EDQ, median
@@ -95,7 +98,7 @@ struct StepParams {
     uint64_t num_chunks;
     uint32_t chunk_elems;
     StepScalars k;
-    EdqPartial* partials;       // one per block, or nullptr
+    EdqFinish fin;              // per-block partials, ticket and record of the EDQ reduction (EDQ kernels)
     EdqPartial* chunk_partials; // one per chunk (per-tensor EDQ), or nullptr
     const uint64_t* replica_bases;  // [num_replicas][num_plan_tensors] base addresses of theta replicas, or nullptr
     int num_replicas;
@@ -357,10 +360,6 @@ __global__ void __launch_bounds__(256) edq_finalize_kernel(const EdqPartial* par
                                                            collage_edq_t* out, int accumulate) {
     __shared__ double s_dot[256], s_sq[256];
     __shared__ unsigned long long s_lost[256];
-    // When launched with programmatic stream serialisation this block may already be resident while
-    // the step kernel runs: wait here until that kernel has completed and its partials are visible.
-    // (A no-op after an ordinary launch.)
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     double d = 0.0, q = 0.0;
     unsigned long long l = 0;
     for (int i = threadIdx.x; i < count; i += 256) {
@@ -383,17 +382,20 @@ __global__ void __launch_bounds__(256) edq_finalize_kernel(const EdqPartial* par
     if (threadIdx.x == 0) {
         double dot = s_dot[0], sq = s_sq[0];
         unsigned long long lost = s_lost[0];
+        unsigned long long fault = 0;
         if (accumulate) {
             dot += out->dot;
             sq += out->sumsq;
             lost += out->lost;
             n += out->n;
+            fault = out->fault;
         }
         out->dot = dot;
         out->sumsq = sq;
         out->edq = sq > 0.0 ? dot / sqrt(sq) : 0.0;
         out->n = n;
         out->lost = lost;
+        out->fault = fault;
     }
 }
 
@@ -431,6 +433,7 @@ __global__ void __launch_bounds__(256) edq_per_tensor_kernel(const EdqPartial* c
         r.edq = s_sq[0] > 0.0 ? s_dot[0] / sqrt(s_sq[0]) : 0.0;
         r.n = sizes[blockIdx.x];
         r.lost = s_lost[0];
+        r.fault = *reinterpret_cast<const volatile unsigned int*>(&g_pipeline_fault);
         out[index[blockIdx.x]] = r;
     }
 }
@@ -450,32 +453,12 @@ __global__ void __launch_bounds__(32) edq_sum_records_kernel(const collage_edq_t
     out->edq = q > 0.0 ? d / sqrt(q) : 0.0;
     out->n = n;
     out->lost = l;
+    out->fault = *reinterpret_cast<const volatile unsigned int*>(&g_pipeline_fault);
 }
 
 void launch_edq_finalize(const EdqPartial* partials, int count, uint64_t n, collage_edq_t* out, cudaStream_t stream,
                          bool accumulate) {
     edq_finalize_kernel<<<1, 256, 0, stream>>>(partials, count, n, out, accumulate ? 1 : 0);
-}
-
-// The same behind a step kernel that has issued griddepcontrol.launch_dependents: the launch is
-// allowed to start before that kernel ends (its first instruction waits for it), which takes the
-// launch latency of this small kernel off the end of every step.
-void launch_edq_finalize_overlapped(const EdqPartial* partials, int count, uint64_t n, collage_edq_t* out,
-                                    cudaStream_t stream, bool accumulate) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(1);
-    cfg.blockDim = dim3(256);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, edq_finalize_kernel, partials, count, n, out, accumulate ? 1 : 0) != cudaSuccess) {
-        (void)cudaGetLastError();
-        edq_finalize_kernel<<<1, 256, 0, stream>>>(partials, count, n, out, accumulate ? 1 : 0);
-    }
 }
 
 // ---------------------------------------------------------------- host side ---
@@ -532,19 +515,22 @@ static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t s
     auto kernel = adamw_step_pipeline_kernel<STRATEGY, EDQ, FLAT, FAST, CONSUMERS, VPT, STAGES, PER_CHUNK, VARIANT>;
     constexpr size_t smem = sizeof(PipeSmem<CONSUMERS, VPT, STAGES, STRATEGY>) + 128;
     constexpr int threads = CONSUMERS + 32;
-    // per instantiation and per device: the shared-memory opt-in is a per-device function attribute
-    static int per_device[64] = {};
+    // per instantiation and per device: the shared-memory opt-in is a per-device function attribute.
+    // Host threads that race on the first call each set the same attribute and store the same number.
+    static std::atomic<int> per_device[64];
     int device = 0;
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return cudaErrorInvalidDevice;
-    if (per_device[device] == 0) {
+    int blocks_per_sm = per_device[device].load(std::memory_order_acquire);
+    if (blocks_per_sm == 0) {
         cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
         if (e != cudaSuccess) return e;
         int b = 0;
         e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, threads, smem);
         if (e != cudaSuccess) return e;
-        per_device[device] = b > 0 ? b : 1;
+        blocks_per_sm = b > 0 ? b : 1;
+        per_device[device].store(blocks_per_sm, std::memory_order_release);
     }
-    uint64_t grid = static_cast<uint64_t>(sm_count) * per_device[device];
+    uint64_t grid = static_cast<uint64_t>(sm_count) * blocks_per_sm;
     if (grid > p.num_chunks) grid = p.num_chunks;
     if (grid > static_cast<uint64_t>(kMaxGrid)) grid = kMaxGrid;
     *grid_out = static_cast<int>(grid);
@@ -613,7 +599,7 @@ static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 // Launches the flat (single tensor) step on device pointers; no-op for n == 0.
 static cudaError_t launch_flat(void* x_hi, void* x_lo, void* m, void* v_hi, void* v_lo, const void* grad, uint64_t n,
-                               const StepScalars& k, int strategy, bool edq, EdqPartial* partials, int sm_count,
+                               const StepScalars& k, int strategy, const EdqFinish& fin, int sm_count,
                                cudaStream_t stream, int* grid_out) {
     *grid_out = 0;
     if (n == 0) return cudaSuccess;
@@ -635,8 +621,8 @@ static cudaError_t launch_flat(void* x_hi, void* x_lo, void* m, void* v_hi, void
     if ((n + chunk - 1) / chunk < 4ull * static_cast<uint64_t>(sm_count)) chunk = tile;
     p.chunk_elems = chunk;
     p.num_chunks = (n + chunk - 1) / chunk;
-    p.partials = partials;
-    return dispatch_step<true>(p, strategy, edq, sm_count, stream, grid_out);
+    p.fin = fin;
+    return dispatch_step<true>(p, strategy, fin.out != nullptr, sm_count, stream, grid_out);
 }
 
 static collage_status_t check_common(const collage_hyper_t* hyper, uint64_t step, int strategy) {
@@ -653,8 +639,30 @@ static collage_status_t check_common(const collage_hyper_t* hyper, uint64_t step
     if (hyper->edq_out) {
         if (!hyper->workspace || hyper->workspace_bytes < kWorkspaceBytes) return COLLAGE_ERR_WORKSPACE;
         if (reinterpret_cast<uintptr_t>(hyper->workspace) & 15u) return COLLAGE_ERR_WORKSPACE;
+        if (reinterpret_cast<uintptr_t>(hyper->edq_out) & 7u) return COLLAGE_ERR_ARG;     // a record of doubles
     }
     return COLLAGE_OK;
+}
+
+// where the pieces of the EDQ reduction live inside a workspace
+static EdqFinish make_finish(void* workspace, void* record, uint64_t n, bool accumulate) {
+    EdqFinish f{};
+    if (record) {
+        f.partials = static_cast<EdqPartial*>(workspace);
+        f.ticket = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + kTicketOffset);
+        f.out = static_cast<collage_edq_t*>(record);
+        f.n = n;
+        f.accumulate = accumulate ? 1 : 0;
+    }
+    return f;
+}
+
+// byte ranges of the EDQ record and workspace of a call, for the overlap checks
+static void push_edq_ranges(std::vector<ByteRange>& ranges, const collage_hyper_t* hyper) {
+    if (hyper->edq_out) {
+        push_bytes(ranges, hyper->edq_out, sizeof(collage_edq_t));
+        push_bytes(ranges, hyper->workspace, kWorkspaceBytes);
+    }
 }
 
 }  // namespace collage
@@ -673,7 +681,7 @@ struct collage_plan {
     int num_given = 0;                   // length of the caller's array
     uint64_t* d_replica_bases = nullptr; // [num_replicas][num_tensors] (non-empty tensors only)
     int num_replicas = 0;
-    std::vector<ByteRange> ranges;       // byte ranges of every array of the plan (overlap checks)
+    std::vector<ByteRange> ranges;       // byte ranges of every array of the plan, sorted by address (overlap checks)
     std::vector<collage_tensor_t> given; // the caller's array, as given
     uint64_t num_chunks = 0;
     uint64_t num_elements = 0;
@@ -725,6 +733,37 @@ collage_status_t collage_derive_scalars(const collage_hyper_t* hyper, uint64_t s
 
 size_t collage_workspace_bytes(uint64_t) { return kWorkspaceBytes; }
 
+collage_status_t collage_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    if (!workspace) return COLLAGE_ERR_NULL;
+    if (workspace_bytes < kWorkspaceBytes || (reinterpret_cast<uintptr_t>(workspace) & 15u)) return COLLAGE_ERR_WORKSPACE;
+    return cudaMemsetAsync(workspace, 0, kWorkspaceBytes, static_cast<cudaStream_t>(stream)) == cudaSuccess ? COLLAGE_OK
+                                                                                                          : COLLAGE_ERR_CUDA;
+}
+
+collage_status_t collage_edq_combine(const collage_edq_t* parts, int count, collage_edq_t* out) {
+    if (!out || (count > 0 && !parts)) return COLLAGE_ERR_NULL;
+    if (count < 0) return COLLAGE_ERR_ARG;
+    collage_edq_t r = {0.0, 0.0, 0.0, 0, 0, 0};
+    for (int i = 0; i < count; ++i) {          // array order: the association of the sums is fixed
+        r.dot += parts[i].dot;
+        r.sumsq += parts[i].sumsq;
+        r.n += parts[i].n;
+        r.lost += parts[i].lost;
+        if (!r.fault) r.fault = parts[i].fault;
+    }
+    r.edq = r.sumsq > 0.0 ? r.dot / std::sqrt(r.sumsq) : 0.0;     // Eq. 3
+    *out = r;
+    return COLLAGE_OK;
+}
+
+const char* collage_build_flavor(void) {
+#ifdef COLLAGE_DATA_MOVEMENT_ONLY
+    return "data-movement-only";
+#else
+    return "product";
+#endif
+}
+
 collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi, void* v_lo, const void* grad,
                                     uint64_t n, const collage_hyper_t* hyper, uint64_t step,
                                     collage_strategy_t strategy, void* stream) {
@@ -738,6 +777,7 @@ collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi,
     for (const void* q : {static_cast<const void*>(x_hi), static_cast<const void*>(x_lo), static_cast<const void*>(m),
                           static_cast<const void*>(v_hi), static_cast<const void*>(v_lo), grad})
         push_range(ranges, q, n);
+    push_edq_ranges(ranges, hyper);
     if (any_overlap(ranges)) return COLLAGE_ERR_ALIAS;
     DeviceInfo dev;
     st = current_device(&dev);
@@ -749,12 +789,11 @@ collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi,
     if (st != COLLAGE_OK) return st;
     const bool edq = hyper->edq_out != nullptr;
     int grid = 0;
-    if (launch_flat(x_hi, x_lo, m, v_hi, v_lo, grad, n, k, strategy, edq, static_cast<EdqPartial*>(hyper->workspace),
+    if (launch_flat(x_hi, x_lo, m, v_hi, v_lo, grad, n, k, strategy, make_finish(hyper->workspace, hyper->edq_out, n, false),
                     dev.sm_count, cs, &grid) != cudaSuccess)
         return COLLAGE_ERR_CUDA;
-    if (edq) {
-        launch_edq_finalize_overlapped(static_cast<EdqPartial*>(hyper->workspace), grid, n,
-                                       static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
+    if (edq && grid == 0) {        // nothing was launched (n == 0): the record still has to say so
+        launch_edq_finalize(static_cast<EdqPartial*>(hyper->workspace), 0, 0, static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
         if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
     return COLLAGE_OK;
@@ -807,7 +846,7 @@ collage_status_t collage_plan_create(const collage_tensor_t* tensors, int num, u
         recs.push_back(r);
         total += t.n;
     }
-    if (any_overlap(ranges)) return COLLAGE_ERR_ALIAS;
+    if (any_overlap(ranges)) return COLLAGE_ERR_ALIAS;     // leaves `ranges` sorted by address
     first_chunk.push_back(chunks.size());
 
     collage_plan* plan = new collage_plan;
@@ -861,6 +900,15 @@ collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const coll
     st = current_device(&dev);
     if (st != COLLAGE_OK) return st;
     if (!plan_on_current_device(plan)) return COLLAGE_ERR_ARG;
+    const bool edq = hyper->edq_out != nullptr;
+    if (edq) {
+        // the record and the workspace may touch neither an array of the plan nor each other
+        std::vector<ByteRange> own;
+        push_edq_ranges(own, hyper);
+        if (any_overlap(own) || overlaps_sorted(plan->ranges, hyper->edq_out, sizeof(collage_edq_t)) ||
+            overlaps_sorted(plan->ranges, hyper->workspace, kWorkspaceBytes))
+            return COLLAGE_ERR_ALIAS;
+    }
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
     StepParams p{};
@@ -870,17 +918,16 @@ collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const coll
     p.chunks = plan->d_chunks;
     p.num_chunks = plan->num_chunks;
     p.chunk_elems = plan->chunk_elems;
-    p.partials = static_cast<EdqPartial*>(hyper->workspace);
+    p.fin = make_finish(hyper->workspace, hyper->edq_out, plan->num_elements, false);
     p.replica_bases = plan->d_replica_bases;
     p.num_replicas = plan->num_replicas;
     p.num_plan_tensors = plan->num_tensors;
-    const bool edq = hyper->edq_out != nullptr;
     int grid = 0;
     if (plan->num_chunks > 0) {
         if (dispatch_step<false>(p, strategy, edq, dev.sm_count, cs, &grid) != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
-    if (edq) {
-        launch_edq_finalize_overlapped(p.partials, grid, plan->num_elements, static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
+    if (edq && grid == 0) {        // an empty plan: the record still has to say so
+        launch_edq_finalize(p.fin.partials, 0, 0, p.fin.out, cs, false);
         if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
     return COLLAGE_OK;
@@ -921,6 +968,23 @@ collage_status_t collage_plan_set_replicas(collage_plan_t* plan, const void* con
     return COLLAGE_OK;
 }
 
+collage_status_t collage_enable_peer_access(int peer_device) {
+    int device = -1, can = 0;
+    if (cudaGetDevice(&device) != cudaSuccess) return COLLAGE_ERR_CUDA;
+    if (peer_device == device || peer_device < 0) return COLLAGE_ERR_ARG;
+    if (cudaDeviceCanAccessPeer(&can, device, peer_device) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return COLLAGE_ERR_ARG;
+    }
+    if (!can) return COLLAGE_ERR_ARG;
+    const cudaError_t e = cudaDeviceEnablePeerAccess(peer_device, 0);
+    if (e == cudaErrorPeerAccessAlreadyEnabled) {
+        (void)cudaGetLastError();          // not an error: clear the runtime's last-error slot
+        return COLLAGE_OK;
+    }
+    return e == cudaSuccess ? COLLAGE_OK : COLLAGE_ERR_CUDA;
+}
+
 size_t collage_plan_workspace_bytes(const collage_plan_t* plan) {
     return plan ? static_cast<size_t>(plan->num_chunks) * sizeof(EdqPartial) + sizeof(EdqPartial) : 0;
 }
@@ -947,6 +1011,18 @@ collage_status_t collage_adamw_step_multi_per_tensor(const collage_plan_t* plan,
     st = current_device(&dev);
     if (st != COLLAGE_OK) return st;
     if (!plan_on_current_device(plan)) return COLLAGE_ERR_ARG;
+    {
+        // the per-tensor records, the chunk workspace and the optional total may touch neither an array
+        // of the plan nor each other
+        std::vector<ByteRange> own;
+        push_bytes(own, per_tensor_out_dev, static_cast<uint64_t>(num) * sizeof(collage_edq_t));
+        push_bytes(own, chunk_workspace, collage_plan_workspace_bytes(plan));
+        push_bytes(own, global_out, sizeof(collage_edq_t));
+        const std::vector<ByteRange> mine = own;
+        if (any_overlap(own)) return COLLAGE_ERR_ALIAS;
+        for (const ByteRange& r : mine)
+            if (overlaps_sorted(plan->ranges, reinterpret_cast<const void*>(r.begin), r.end - r.begin)) return COLLAGE_ERR_ALIAS;
+    }
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
 
     StepParams p{};
@@ -1005,14 +1081,14 @@ collage_status_t collage_pipeline_fault(uint32_t* out_host) {
 namespace collage {
 // One warp waits on a barrier that nothing completes, with a short bound; the wait runs out, the
 // code 100 goes to the fault word and the kernel returns in the ordinary way.
-__global__ void __launch_bounds__(32) wait_timeout_kernel(long long limit_cycles) {
+__global__ void __launch_bounds__(32) wait_timeout_kernel(unsigned long long limit_ns) {
     __shared__ alignas(8) uint64_t bar;
     if (threadIdx.x == 0) {
         pipe::mbar_init(&bar, 1);
         pipe::mbar_init_fence();
     }
     __syncwarp();
-    (void)__all_sync(0xFFFFFFFFu, pipe::mbar_wait(&bar, 0u, 99u, &g_pipeline_fault, limit_cycles));
+    (void)__all_sync(0xFFFFFFFFu, pipe::mbar_wait(&bar, 0u, 99u, &g_pipeline_fault, limit_ns));
 }
 }  // namespace collage
 
@@ -1021,7 +1097,7 @@ collage_status_t collage_wait_timeout_selftest(uint32_t limit_ms, void* stream) 
     DeviceInfo dev;
     const collage_status_t st = current_device(&dev);
     if (st != COLLAGE_OK) return st;
-    wait_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<long long>(limit_ms) * 2000000LL);
+    wait_timeout_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<unsigned long long>(limit_ms) * 1000000ULL);
     return cudaGetLastError() == cudaSuccess ? COLLAGE_OK : COLLAGE_ERR_CUDA;
 }
 
@@ -1035,9 +1111,13 @@ struct HostStepContext {
     bool ready = false;
 };
 
-// Two copy streams and a handful of events per device, created on the first staged call.
+// Two copy streams and a handful of events per device, created on the first staged call (under a
+// lock: two host threads may make that call together).
 cudaError_t host_step_context(int device, HostStepContext** out) {
     static HostStepContext ctx[64];
+    static std::mutex guard;
+    if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> hold(guard);
     HostStepContext& c = ctx[device];
     if (!c.ready) {
         cudaError_t e;
@@ -1074,7 +1154,7 @@ collage_status_t collage_adamw_step_host(void* x_hi, void* x_lo, void* m, void* 
         push_range(ranges, q, n);
     if (any_overlap(ranges)) return COLLAGE_ERR_ALIAS;
 
-    // staging layout: [record 256 B][EDQ partials][2 slabs x 6 arrays x slab_elems bfloat16]
+    // staging layout: [record 256 B][EDQ workspace][2 slabs x 6 arrays x slab_elems bfloat16]
     const size_t fixed = 256 + kWorkspaceBytes;
     if (!staging_dev || (reinterpret_cast<uintptr_t>(staging_dev) & 255u) || staging_bytes < fixed + 2 * 6 * 2 * 16384)
         return COLLAGE_ERR_WORKSPACE;
@@ -1101,7 +1181,10 @@ collage_status_t collage_adamw_step_host(void* x_hi, void* x_lo, void* m, void* 
     const bool edq = edq_host != nullptr;
 #define COLLAGE_TRY(call) do { if ((call) != cudaSuccess) return COLLAGE_ERR_CUDA; } while (0)
 
-    if (edq) COLLAGE_TRY(cudaMemsetAsync(record, 0, sizeof(collage_edq_t), cs));
+    if (edq) {
+        COLLAGE_TRY(cudaMemsetAsync(record, 0, sizeof(collage_edq_t), cs));
+        COLLAGE_TRY(cudaMemsetAsync(reinterpret_cast<char*>(partials) + kTicketOffset, 0, 64, cs));   // the staging buffer is ours to clear
+    }
     COLLAGE_TRY(cudaEventRecord(c->start, cs));               // copies start after the caller's earlier work
     COLLAGE_TRY(cudaStreamWaitEvent(c->in, c->start, 0));
     const uint64_t nslabs = (n + slab - 1) / slab;
@@ -1117,12 +1200,8 @@ collage_status_t collage_adamw_step_host(void* x_hi, void* x_lo, void* m, void* 
         COLLAGE_TRY(cudaStreamWaitEvent(cs, c->loaded[b], 0));
         int grid = 0;
         COLLAGE_TRY(launch_flat(dev_array(b, 0), x_lo ? dev_array(b, 1) : nullptr, dev_array(b, 2), dev_array(b, 3),
-                                v_lo ? dev_array(b, 4) : nullptr, dev_array(b, 5), len, k, strategy, edq, partials,
-                                dev.sm_count, cs, &grid));
-        if (edq) {
-            launch_edq_finalize_overlapped(partials, grid, len, record, cs, true);
-            COLLAGE_TRY(cudaGetLastError());
-        }
+                                v_lo ? dev_array(b, 4) : nullptr, dev_array(b, 5), len, k, strategy,
+                                make_finish(partials, edq ? record : nullptr, len, true), dev.sm_count, cs, &grid));
         COLLAGE_TRY(cudaEventRecord(c->computed[b], cs));
         COLLAGE_TRY(cudaStreamWaitEvent(c->out, c->computed[b], 0));
         for (int a = 0; a < 5; ++a)

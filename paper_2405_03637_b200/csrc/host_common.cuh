@@ -2,6 +2,7 @@
 // double -> bfloat16 rounding used for the step's scalars, and the EDQ partial-sum layout.
 #pragma once
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdint>
 #include <cstring>
@@ -19,33 +20,35 @@ struct EdqPartial {
     unsigned long long lost, pad;
 };
 constexpr int kMaxGrid = 4096;                       // upper bound on persistent grid size
-constexpr size_t kWorkspaceBytes = sizeof(EdqPartial) * kMaxGrid;
+// workspace layout: kMaxGrid partials, then the ticket counter of the last-block reduction
+constexpr size_t kTicketOffset = sizeof(EdqPartial) * kMaxGrid;
+constexpr size_t kWorkspaceBytes = kTicketOffset + 64;
 
 struct DeviceInfo {
     int sm_count = 0;
     int cc_major = 0;
-    bool known = false;
 };
 
 // Facts about the current device, looked up once per device.  Returns COLLAGE_ERR_ARCH unless
 // the device is compute capability 10.x: the kernels are built for sm_100a only and there is
-// no fallback.
+// no fallback.  Safe to call from several host threads at once: the cached word is written with
+// one atomic store after the (idempotent) lookup, so racing first calls store the same value.
 inline collage_status_t current_device(DeviceInfo* out) {
-    static DeviceInfo cache[64];
+    static std::atomic<uint32_t> cache[64];            // 0 = unknown, else 1 | sm_count << 1 | cc_major << 17
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return COLLAGE_ERR_CUDA;
     if (dev < 0 || dev >= 64) return COLLAGE_ERR_CUDA;
-    DeviceInfo& d = cache[dev];
-    if (!d.known) {
+    uint32_t w = cache[dev].load(std::memory_order_acquire);
+    if (w == 0) {
         int sm = 0, major = 0;
         if (cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return COLLAGE_ERR_CUDA;
         if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return COLLAGE_ERR_CUDA;
-        d.sm_count = sm;
-        d.cc_major = major;
-        d.known = true;
+        w = 1u | (static_cast<uint32_t>(sm & 0xFFFF) << 1) | (static_cast<uint32_t>(major & 0xFF) << 17);
+        cache[dev].store(w, std::memory_order_release);
     }
-    *out = d;
-    return d.cc_major == 10 ? COLLAGE_OK : COLLAGE_ERR_ARCH;
+    out->sm_count = static_cast<int>((w >> 1) & 0xFFFF);
+    out->cc_major = static_cast<int>((w >> 17) & 0xFF);
+    return out->cc_major == 10 ? COLLAGE_OK : COLLAGE_ERR_ARCH;
 }
 
 // Byte ranges [begin, end) of the arrays of one call; overlap of any two is an error.
@@ -55,6 +58,19 @@ struct ByteRange {
 
 inline void push_range(std::vector<ByteRange>& v, const void* p, uint64_t n_elems) {
     if (p && n_elems) v.push_back({reinterpret_cast<uintptr_t>(p), reinterpret_cast<uintptr_t>(p) + 2 * n_elems});
+}
+
+inline void push_bytes(std::vector<ByteRange>& v, const void* p, uint64_t bytes) {
+    if (p && bytes) v.push_back({reinterpret_cast<uintptr_t>(p), reinterpret_cast<uintptr_t>(p) + bytes});
+}
+
+// Does [p, p + bytes) overlap any range of `sorted` (sorted by begin, pairwise disjoint)?
+inline bool overlaps_sorted(const std::vector<ByteRange>& sorted, const void* p, uint64_t bytes) {
+    if (!p || !bytes || sorted.empty()) return false;
+    const uintptr_t b = reinterpret_cast<uintptr_t>(p), e = b + bytes;
+    // first range that begins at or after e; the one before it is the only candidate that can reach past b
+    auto it = std::lower_bound(sorted.begin(), sorted.end(), e, [](const ByteRange& r, uintptr_t x) { return r.begin < x; });
+    return it != sorted.begin() && (it - 1)->end > b;
 }
 
 inline bool any_overlap(std::vector<ByteRange>& v) {

@@ -12,13 +12,16 @@
 //
 // Tiles that cannot be bulk-copied (tensor not 16-byte aligned, or the ragged last tile of a
 // tensor) flow through the same barriers but are processed straight from global memory.
-// Every wait is bounded: after ~2 s a thread records a fault in g_pipeline_fault and leaves.
+// Every wait is bounded: after two seconds a thread records a fault in g_pipeline_fault and leaves.
+// EDQ: float within a vector, double per thread, fixed-order tree per block, one partial per block;
+// the block that finishes last adds the partials (edq_reduce.cuh), so a step is one launch.
 //
 // On the host-validated lean chain (FAST) a consumer runs the branch-free compute_vec_fast on its
 // 8 parameters; a vector with a lane that chain cannot answer is repeated in place, from the tile
 // that still holds its inputs, by the out-of-line careful_vector_in_tile.
 #pragma once
 #include "bulk_pipe.cuh"
+#include "edq_reduce.cuh"
 #include "mcf_device.cuh"
 
 namespace collage {
@@ -59,6 +62,7 @@ struct PipeSmem {
     alignas(8) uint64_t red_full, red_free;   // hand-over of per-chunk EDQ sums (PER_CHUNK only)
     double red_dot[CONSUMERS / 32], red_sq[CONSUMERS / 32];
     unsigned long long red_lost[CONSUMERS / 32];
+    EdqFinishSmem finish;                     // the last block's sum over all blocks (EDQ, not PER_CHUNK)
 };
 
 // PER_CHUNK: the EDQ sums are written once per chunk (p.chunk_partials[chunk]) instead of once per
@@ -74,8 +78,6 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
     using Smem = PipeSmem<CONSUMERS, VPT, STAGES, STRATEGY>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 127) & ~static_cast<uintptr_t>(127));
 
-    // the small kernel that sums the EDQ partials may be launched now; it waits for this grid to end
-    if (EDQ && !PER_CHUNK) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const bool is_producer = threadIdx.x >= CONSUMERS;
     if (threadIdx.x == 0) {
 #pragma unroll
@@ -325,17 +327,18 @@ adamw_step_pipeline_kernel(const __grid_constant__ StepParams p) {
             }
         }
         __syncthreads();
+        double d = 0.0, q = 0.0;
+        unsigned long long l = 0;
         if (threadIdx.x == 0) {
-            double d = 0.0, q = 0.0;
-            unsigned long long l = 0;
 #pragma unroll
             for (int w = 0; w < kWarps; ++w) {
                 d += sm.red_dot[w];
                 q += sm.red_sq[w];
                 l += sm.red_lost[w];
             }
-            p.partials[blockIdx.x] = EdqPartial{d, q, l, 0ull};
         }
+        // one partial per block; the block that finishes last adds them up and writes the record
+        edq_publish_and_finish(p.fin, sm.finish, d, q, l, &g_pipeline_fault);
     }
 }
 

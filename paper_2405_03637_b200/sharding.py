@@ -6,8 +6,6 @@ quantity is EDQ (Eq. 3), whose two sums -- and the lost-update count -- are adde
 """
 from __future__ import annotations
 
-import math
-
 
 def partition(sizes: list[int], world: int, align: int = 8) -> list[list[tuple[int, int, int]]]:
     """Split tensors of the given sizes over `world` ranks.
@@ -75,11 +73,90 @@ def replica_rows(peer_x_hi, ranges):
 
 
 def allreduce_edq(sums, dist=None, group=None) -> dict:
-    """Add {dot, sumsq, lost} over ranks in place (a 3-element float64 tensor) and form EDQ.
+    """Add {dot, sumsq, lost} over ranks in place (a 3-element float64 tensor); the library forms EDQ.
 
-    `dist` is torch.distributed (NCCL on GPUs, gloo on CPU); None means a single process.
+    `dist` is torch.distributed (NCCL on GPUs, gloo on CPU); None means a single process.  The
+    quotient of Eq. 3 is taken by the library's `collage_edq_combine` on the summed record, not here.
     """
+    from . import binding
     if dist is not None and dist.is_initialized() and dist.get_world_size(group) > 1:
         dist.all_reduce(sums, group=group)
     dot, sumsq, lost = (float(x) for x in sums.tolist())
-    return dict(dot=dot, sumsq=sumsq, edq=dot / math.sqrt(sumsq) if sumsq > 0 else 0.0, lost=int(round(lost)))
+    return binding.edq_combine([dict(dot=dot, sumsq=sumsq, lost=int(round(lost)))])
+
+
+# --------------------------------------------------------------- harness ---
+# One rank of the sharded step, independent of where the memory lives: the benchmark builds it on
+# CUDA tensors (peer copies mapped through CUDA IPC), the CPU test on shared-memory CPU tensors with
+# the oracle as the stepper.  The exchange pattern is the library's: a rank steps its slice and the
+# new theta of that slice is stored into every rank's full copy; {dot, sumsq, lost} are all-reduced.
+
+class ShardedRank:
+    """State, plan rows and replica table of rank `rank` out of `world`.
+
+    theta_copies[r][i] : tensor i of rank r's full copy of theta, as mapped into this process
+                         (theta_copies[rank] is this rank's own copy; the others are peer memory)
+    alloc(n)           : a zeroed bfloat16 tensor of n elements where this rank keeps optimizer state
+    """
+
+    def __init__(self, sizes, rank, world, theta_copies, alloc, strategy):
+        self.sizes, self.rank, self.world, self.strategy = list(sizes), rank, world, strategy
+        self.ranges = partition(self.sizes, world)[rank]
+        full = [(theta_copies[rank][i], None, None, None, None, None) for i in range(len(self.sizes))]
+        self.rows = []
+        for (i, b, e), cut in zip(self.ranges, slice_rows(full, self.ranges)):
+            n = e - b
+            self.rows.append((cut[0], alloc(n) if strategy >= 1 else None, alloc(n), alloc(n),
+                              alloc(n) if strategy in (2, 4) else None, alloc(n), n))
+        peers = [theta_copies[r] for r in range(world) if r != rank]
+        self.replicas = replica_rows(peers, self.ranges)
+        self.elements = sum(r[6] for r in self.rows)
+
+    def gathered_bytes_per_step(self) -> int:
+        """Bytes this rank sends to peers per step: 2 B per owned parameter and peer."""
+        return 2 * self.elements * (self.world - 1)
+
+
+class CudaStepper:
+    """Steps a ShardedRank with the library: one multi-tensor launch that also stores theta to the peers."""
+
+    def __init__(self, shard: ShardedRank, torch):
+        from . import binding
+        self.B, self.shard, self.torch = binding, shard, torch
+        device = shard.rows[0][0].device if shard.rows else torch.device("cuda")
+        self.plan = binding.plan_create(shard.rows)
+        if shard.replicas:
+            binding.plan_set_replicas(self.plan, shard.replicas)
+        self.record = torch.zeros(64, dtype=torch.uint8, device=device)
+        self.workspace = torch.empty(binding.workspace_bytes(), dtype=torch.uint8, device=device)
+        binding.workspace_init(self.workspace)
+        # what ranks exchange: {dot, sumsq} as doubles and the lost count, views of the device record
+        self.sums = self.record[:16].view(torch.float64)
+        self.lost = self.record[32:40].view(torch.int64)
+
+    def step(self, hyp: dict, t: int, stream=None):
+        B = self.B
+        B.adamw_step_multi(self.plan, B.make_hyper(**hyp, edq_out=self.record, workspace=self.workspace), t,
+                           self.shard.strategy, stream)
+
+    def allreduce(self, dist):
+        """Sum the EDQ partial sums over ranks on the device (no host synchronisation)."""
+        if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+            dist.all_reduce(self.sums)
+            dist.all_reduce(self.lost)
+
+    def read(self) -> dict:
+        """The record after `allreduce`: Eq. 3 on the summed sums, formed by the library."""
+        rec = self.B.read_edq(self.record)
+        return self.B.edq_combine([dict(dot=rec["dot"], sumsq=rec["sumsq"], lost=rec["lost"], fault=rec["fault"])])
+
+    def close(self):
+        self.B.plan_destroy(self.plan)
+
+
+def theta_checksum(copy, torch) -> int:
+    """Order-independent digest of a full theta copy (sum of the bit patterns), to compare copies across ranks."""
+    total = 0
+    for t in copy:
+        total += int(t.view(torch.int16).to(torch.int64).sum().item())
+    return total

@@ -28,6 +28,15 @@ def pytest_collection_modifyitems(config, items):
             item.add_marker(skip)
 
 
+@pytest.fixture(scope="session", autouse=True)
+def library_under_test_is_the_product_build():
+    """Every test runs against the ordinary in-tree build, never a measurement build of the same sources."""
+    from paper_2405_03637_b200 import binding, build
+    build.build()
+    assert binding.build_flavor() == "product"
+    assert Path(binding.lib()._name) == ROOT / "paper_2405_03637_b200" / "libcollage_b200.so"
+
+
 def bf16_window(e_lo: int, e_hi: int, signs=(0, 1), with_zero=False) -> np.ndarray:
     """All bfloat16 bit patterns whose unbiased exponent is in [e_lo, e_hi] (normal numbers)."""
     out = []

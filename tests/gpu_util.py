@@ -58,6 +58,7 @@ class EdqBuffers:
     def __init__(self, device="cuda"):
         self.out = torch.zeros(64, dtype=torch.uint8, device=device)
         self.ws = torch.empty(B.workspace_bytes(), dtype=torch.uint8, device=device)
+        B.workspace_init(self.ws)                 # once; every step leaves it ready for the next
 
     def hyper(self, hyp: dict, flags=0) -> B.Hyper:
         return B.make_hyper(hyp["lr"], hyp["beta1"], hyp["beta2"], hyp["eps"], hyp["weight_decay"], flags,

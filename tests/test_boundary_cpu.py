@@ -31,7 +31,7 @@ def test_library_exports_every_declared_symbol(L):
 
 def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(B.Hyper) == 5 * 8 + 8 + 3 * 8        # flags padded to 8
-    assert ctypes.sizeof(B.Edq) == 40
+    assert ctypes.sizeof(B.Edq) == 48 == B.EDQ_RECORD_BYTES
     assert ctypes.sizeof(B.Tensor) == 56
     assert B.workspace_bytes(0) == B.workspace_bytes(1 << 40) > 0
 
@@ -100,6 +100,20 @@ def test_argument_errors_are_reported_before_any_cuda_call(L):
     assert call(hyper=h) == B.ERR_WORKSPACE
     h.workspace, h.workspace_bytes = dummy * 8, 16
     assert call(hyper=h) == B.ERR_WORKSPACE
+    # the record and the workspace may overlap neither a tensor nor each other
+    big = B.workspace_bytes()
+    h.workspace, h.workspace_bytes = dummy * 8, big
+    h.edq_out = dummy + 8                                              # inside x_hi
+    assert call(hyper=h) == B.ERR_ALIAS
+    h.edq_out, h.workspace = dummy * 7, dummy * 3 - 64                 # workspace runs into v_hi
+    assert call(hyper=h) == B.ERR_ALIAS
+    h.edq_out, h.workspace = dummy * 8 + 4096, dummy * 8               # record inside the workspace
+    assert call(hyper=h) == B.ERR_ALIAS
+    h.edq_out, h.workspace = dummy * 7 + 4, dummy * 8                  # a record of doubles must be 8-byte aligned
+    assert call(hyper=h) == B.ERR_ARG
+    assert L.collage_workspace_init(None, big, None) == B.ERR_NULL
+    assert L.collage_workspace_init(dummy, 16, None) == B.ERR_WORKSPACE
+    assert L.collage_workspace_init(dummy + 4, big, None) == B.ERR_WORKSPACE
     # derive_scalars
     out = (ctypes.c_uint16 * 11)()
     assert L.collage_derive_scalars(None, 1, out) == B.ERR_NULL
@@ -128,6 +142,49 @@ def test_argument_errors_are_reported_before_any_cuda_call(L):
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "_lib", None)
-    monkeypatch.setattr(B, "_LIB_PATH", tmp_path / "absent.so")
+    monkeypatch.setattr(B, "_lib_path", tmp_path / "absent.so")
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         B.lib()
+
+
+def test_no_environment_variable_selects_the_library(monkeypatch, tmp_path):
+    # the library that runs is the in-tree build unless load(path) is called; load() after first use is refused
+    monkeypatch.setenv("COLLAGE_B200_LIB", str(tmp_path / "elsewhere.so"))
+    assert B.lib()._name == str(ROOT / "paper_2405_03637_b200" / "libcollage_b200.so")
+    assert B.build_flavor() == "product"
+    with pytest.raises(RuntimeError, match="already loaded"):
+        B.load(tmp_path / "elsewhere.so")
+
+
+def test_edq_combine_is_equation_3_on_the_summed_partial_sums(L):
+    # records of disjoint slices of one step, as ranks or tensors would hold them, against the oracle's sums
+    # over the whole array; the quotient is taken by the library, on the host, with no CUDA call
+    import numpy as np
+    from paper_2405_03637_b200 import workloads as W
+    n = 50_000
+    th = W.bits(W.flat_weights(n, 40)); g = W.bits(W.flat_grads(n, 40, 1))
+    hyp = dict(lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
+    z = lambda: np.zeros(n, np.uint16)
+    whole_state = [th.copy(), z(), z(), z()]
+    whole, _ = oracle.adamw_step(whole_state[0], None, whole_state[1], whole_state[2], None, g, step=1, strategy=0, **hyp)
+    cuts, parts = [0, 7, 12_345, 12_345, 40_000, n], []
+    for lo, hi in zip(cuts, cuts[1:]):
+        st = [th[lo:hi].copy(), np.zeros(hi - lo, np.uint16), np.zeros(hi - lo, np.uint16)]
+        s, _ = oracle.adamw_step(st[0], None, st[1], st[2], None, g[lo:hi].copy(), step=1, strategy=0, **hyp)
+        parts.append(dict(s, n=hi - lo))
+    got = B.edq_combine(parts)
+    assert got["n"] == n and got["lost"] == whole["lost"] and got["fault"] == 0
+    assert got["dot"] == pytest.approx(whole["dot"], rel=1e-12) and got["sumsq"] == pytest.approx(whole["sumsq"], rel=1e-12)
+    assert got["edq"] == pytest.approx(whole["edq"], rel=1e-12)
+    assert got["edq"] == got["dot"] / np.sqrt(got["sumsq"])
+    # fixed order: the sums are those of a left-to-right addition
+    d = 0.0
+    for p in parts:
+        d += p["dot"]
+    assert got["dot"] == d
+    assert B.edq_combine([]) == dict(dot=0.0, sumsq=0.0, edq=0.0, n=0, lost=0, fault=0)
+    assert B.edq_combine([dict(dot=1.0, sumsq=0.0, lost=0)])["edq"] == 0.0                     # zero norm: EDQ is 0
+    assert B.edq_combine([dict(dot=0.0, sumsq=1.0, lost=0, fault=0), dict(dot=0.0, sumsq=1.0, lost=0, fault=41)])["fault"] == 41
+    assert L.collage_edq_combine(None, 1, ctypes.byref(B.Edq())) == B.ERR_NULL
+    assert L.collage_edq_combine(None, 0, None) == B.ERR_NULL
+    assert L.collage_edq_combine(None, -1, ctypes.byref(B.Edq())) == B.ERR_ARG

@@ -123,7 +123,7 @@ def test_per_tensor_edq_matches_oracle_tensor_by_tensor(strategy, chunk):
     host, dev, grads, rows = _build(shapes, strategy, seed=7, misalign_of=lambda i: (0, 1, 0)[i % 3])
     plan = B.plan_create(rows, chunk)
     num = len(shapes)
-    per = torch.zeros(num * 40, dtype=torch.uint8, device="cuda")
+    per = torch.zeros(num * B.EDQ_RECORD_BYTES, dtype=torch.uint8, device="cuda")
     cws = torch.empty(B.plan_workspace_bytes(plan), dtype=torch.uint8, device="cuda")
     assert B.plan_workspace_bytes(plan) >= 32 * B.plan_num_chunks(plan)
     total = torch.zeros(64, dtype=torch.uint8, device="cuda")
@@ -136,7 +136,7 @@ def test_per_tensor_edq_matches_oracle_tensor_by_tensor(strategy, chunk):
         tot = dict(dot=0.0, sumsq=0.0, lost=0)
         for i, (st, g) in enumerate(zip(host, gbits)):
             if g.size == 0:
-                assert recs[i] == dict(dot=0.0, sumsq=0.0, edq=0.0, n=0, lost=0)
+                assert recs[i] == dict(dot=0.0, sumsq=0.0, edq=0.0, n=0, lost=0, fault=0)
                 continue
             want = oracle_step(st, g, t, strategy, hyp, threads=1)
             edq_close(recs[i], want)

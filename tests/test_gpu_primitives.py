@@ -186,7 +186,7 @@ def test_standalone_edq_matches_oracle():
             assert abs(got[k] - want[k]) <= 1e-5 * abs(want[k])
         assert got["lost"] == want["lost"] and got["n"] == n
         if has_lo:
-            assert got["lost"] >= kp.size + n // 7 - kp.size // 7 - 2
+            assert got["lost"] >= kp.size                      # every planted pair is counted
 
 
 def test_standalone_edq_past_2_to_32_elements_is_the_sum_of_its_pieces():

@@ -104,6 +104,72 @@ def test_two_ranks_reproduce_the_global_edq():
     assert sum(c for _, _, c in results) == checksum                  # the slices together are the whole state
 
 
+def _as_u16(t):
+    """numpy uint16 view of a CPU bfloat16 tensor (shares its memory)."""
+    return t.view(torch.int16).numpy().view(np.uint16)
+
+
+def _harness_rank(rank, world, port, sizes, copies, out_q):
+    # the benchmark's sharded flow on CPU: the same ShardedRank (partition, plan rows, replica table) and the
+    # same all-reduce helper; the oracle steps the rows, and a plain copy into the peers' shared-memory theta
+    # stands in for the step kernel's replica stores
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        hyp, strategy = W.HYPERS, 2
+        alloc = lambda n: torch.zeros(n, dtype=torch.bfloat16)
+        shard = sharding.ShardedRank(sizes, rank, world, copies, alloc, strategy)
+        assert len(shard.replicas) == world - 1 and all(len(rep) == len(shard.rows) for rep in shard.replicas)
+        assert shard.gathered_bytes_per_step() == 2 * shard.elements * (world - 1)
+        for t in (1, 2):
+            sums = torch.zeros(3, dtype=torch.float64)
+            for k, ((i, b, e), row) in enumerate(zip(shard.ranges, shard.rows)):
+                g = W.bits(W.flat_grads(sizes[i], 700 + i, t))[b:e]
+                x_hi, x_lo, m, v_hi, v_lo = (_as_u16(a) for a in row[:5])
+                s, _ = oracle.adamw_step(x_hi, x_lo, m, v_hi, v_lo, g, step=t, strategy=strategy, **hyp)
+                sums += torch.tensor([s["dot"], s["sumsq"], float(s["lost"])], dtype=torch.float64)
+                for rep in shard.replicas:                       # theta of the slice goes to every peer's copy
+                    rep[k].copy_(row[0])
+            got = sharding.allreduce_edq(sums, dist)             # also the point after which every copy is complete
+            dist.barrier()
+        out_q.put((rank, got, sharding.theta_checksum(copies[rank], torch)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_drive_the_sharded_harness_with_the_oracle_as_stepper():
+    sizes = [50_001, 4096, 9, 120_000, 8]
+    world = 2
+    theta = [W.flat_weights(n, 700 + i) for i, n in enumerate(sizes)]
+    copies = [[t.clone().share_memory_() for t in theta] for _ in range(world)]     # each rank's full copy of theta
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_harness_rank, args=(r, world, port, sizes, copies, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = [q.get(timeout=180) for _ in procs]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    # the unsharded step over the whole set
+    tot, full = dict(dot=0.0, sumsq=0.0, lost=0), []
+    for i, n in enumerate(sizes):
+        st = [W.bits(theta[i]), *(np.zeros(n, np.uint16) for _ in range(4))]
+        for t in (1, 2):
+            s, _ = oracle.adamw_step(st[0], st[1], st[2], st[3], st[4], W.bits(W.flat_grads(n, 700 + i, t)), step=t,
+                                     strategy=2, **W.HYPERS)
+        tot["dot"] += s["dot"]; tot["sumsq"] += s["sumsq"]; tot["lost"] += s["lost"]
+        full.append(st[0])
+    for r in range(world):                                            # every rank's copy holds the whole new theta
+        for i in range(len(sizes)):
+            assert np.array_equal(_as_u16(copies[r][i]), full[i]), (r, i)
+    want = sharding.theta_checksum([W.from_bits(f) for f in full], torch)
+    for rank, got, checksum in results:
+        assert checksum == want
+        assert got["edq"] == pytest.approx(tot["dot"] / np.sqrt(tot["sumsq"]), rel=1e-12) and got["lost"] == tot["lost"]
+
+
 def test_slices_of_all_ranks_tile_every_tensor_and_keep_alignment():
     sizes = [4096, 9, 100_003, 0, 65_536]
     rows = []

@@ -28,7 +28,8 @@ def _inputs(n, seed):
     new_hi[::5] = old_hi[::5]
     new_lo[::5] = old_lo[::5]                                   # some updates lost entirely
     to_dev = lambda a: torch.from_numpy(a.view(np.int16).copy()).view(torch.bfloat16).cuda()
-    return [to_dev(a) for a in (old_hi, old_lo, new_hi, new_lo, delta)]
+    host = (old_hi, old_lo, new_hi, new_lo, delta)
+    return [to_dev(a) for a in host], host
 
 
 def _close(got, want):
@@ -44,12 +45,15 @@ def test_static_scratch_matches_workspace_version_on_two_calls_in_a_row():
     # two different problems back to back through the one shared array: the second call must not see
     # anything of the first (a larger problem first, so stale partial sums would be left behind)
     for n, seed, with_lo in [(5_000_003, 1, True), (2_097_153, 2, False)]:
-        old_hi, old_lo, new_hi, new_lo, delta = _inputs(n, seed)
+        (old_hi, old_lo, new_hi, new_lo, delta), host = _inputs(n, seed)
         lo_args = (old_lo, new_lo) if with_lo else (None, None)
         B.edq(old_hi, lo_args[0], new_hi, lo_args[1], delta, n, ref_out, ws)
         B.edq_static(old_hi, lo_args[0], new_hi, lo_args[1], delta, n, out)
         torch.cuda.synchronize()
         _close(B.read_edq(out), B.read_edq(ref_out))
+        # and against the CPU oracle directly (Eq. 2-3 in double, index order)
+        want = oracle.edq(host[0], host[1] if with_lo else None, host[2], host[3] if with_lo else None, host[4])
+        _close(B.read_edq(out), dict(want, n=n))
     # same inputs again: identical result (deterministic, nothing carried over)
     first = B.read_edq(out)
     B.edq_static(old_hi, None, new_hi, None, delta, n, out)
@@ -63,6 +67,27 @@ def test_static_scratch_matches_workspace_version_on_two_calls_in_a_row():
     B.edq_static(old_hi, None, new_hi, None, delta, 0, out)
     torch.cuda.synchronize()
     assert B.read_edq(out)["edq"] == 0.0 and B.read_edq(out)["n"] == 0
+
+
+def test_calls_leave_the_amount_of_free_device_memory_unchanged():
+    # what the entry point exists for: it takes no device memory.  The first call on a device looks the
+    # scratch array's address up (and the CUDA runtime may load the library's code then); from the second
+    # call on, free memory as the driver reports it is the same before and after any number of calls,
+    # small and large, with and without second components.
+    (old_hi, old_lo, new_hi, new_lo, delta), host = _inputs(3_000_001, 3)
+    out = torch.zeros(64, dtype=torch.uint8, device="cuda")
+    B.edq_static(old_hi, old_lo, new_hi, new_lo, delta, 1000, out)
+    B.edq_static(old_hi, None, new_hi, None, delta, 1000, out)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for n in (1, 2049, 300_000, 3_000_001):
+        B.edq_static(old_hi, old_lo, new_hi, new_lo, delta, n, out)
+        B.edq_static(old_hi, None, new_hi, None, delta, n, out)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    want = oracle.edq(host[0], None, host[2], None, host[4])
+    _close(B.read_edq(out), dict(want, n=3_000_001))
 
 
 def test_sizes_beyond_the_capacity_are_rejected():
