@@ -496,7 +496,7 @@ def run_e2e(torch, B, W, device, args):
     torch.cuda.synchronize()
     wall = time.perf_counter() - t0
     ms = max(e0.elapsed_time(e1), wall * 1e3) / steps
-    return {"value": n / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 12 * n, "d2h_bytes_per_step": 10 * n + 40,
+    return {"value": n / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": 12 * n, "d2h_bytes_per_step": 10 * n + 48,
             "ms_per_step": ms, "steps": steps,
             "sample": f"first {n} parameters of the flattened workload, state in pinned host memory, "
                       "collage_adamw_step_host (768 MiB device staging)"}

@@ -85,6 +85,13 @@ typedef enum {
  *   Adam part (-a) (*) r.  A, B, C.  EDQ then measures against d + update. */
 #define COLLAGE_FLAG_TWOSUM_GROW 2u
 #define COLLAGE_FLAG_DECAY_BY_GROW 4u
+/* Which kernel steps a flat tensor (collage_adamw_step, collage_adamw_step_host).  By default the size
+ * decides: up to 2^21 parameters a kernel without staging, one 8-parameter vector per thread straight
+ * from global memory (shortest latency); above, the bulk-copy pipeline that streams at HBM bandwidth.
+ * Both compute the same bits.  These flags pin the choice (tests and measurements); setting both is
+ * ERR_ARG; entry points without such a choice ignore them. */
+#define COLLAGE_FLAG_PIPELINE_KERNEL 8u
+#define COLLAGE_FLAG_DIRECT_KERNEL 16u
 
 /* Hyper-parameters of one step (Algorithm 2 line 1).  HOST struct.
  * Valid ranges: lr, eps, weight_decay >= 0 and finite; 0 <= beta1, beta2 < 1. */

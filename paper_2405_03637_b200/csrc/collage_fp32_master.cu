@@ -340,7 +340,8 @@ extern "C" collage_status_t collage_adamw_step_fp32(void* theta, void* master, v
                                                     void* stream) {
     if (!hyper) return COLLAGE_ERR_NULL;
     if (step == 0 || !hyper_in_range(hyper)) return COLLAGE_ERR_ARG;
-    if (hyper->flags & ~COLLAGE_FLAG_EPS_INSIDE_SQRT) return COLLAGE_ERR_ARG;
+    if (hyper->flags & ~(COLLAGE_FLAG_EPS_INSIDE_SQRT | COLLAGE_FLAG_PIPELINE_KERNEL | COLLAGE_FLAG_DIRECT_KERNEL))
+        return COLLAGE_ERR_ARG;                               // the kernel-choice flags mean nothing here and are ignored
     if (hyper->edq_out) {
         if (!hyper->workspace || hyper->workspace_bytes < kWorkspaceBytes ||
             (reinterpret_cast<uintptr_t>(hyper->workspace) & 15u))
@@ -388,7 +389,7 @@ extern "C" collage_status_t collage_adamw_step_fp32(void* theta, void* master, v
     p.k.neg_a = -static_cast<float>(hyper->lr);
     p.k.lam = static_cast<float>(hyper->weight_decay);
     p.k.eps = static_cast<float>(hyper->eps);
-    p.k.flags = hyper->flags;
+    p.k.flags = hyper->flags & COLLAGE_FLAG_EPS_INSIDE_SQRT;
     if (hyper->edq_out) {
         p.fin.partials = static_cast<EdqPartial*>(hyper->workspace);
         p.fin.ticket = reinterpret_cast<unsigned int*>(static_cast<char*>(hyper->workspace) + kTicketOffset);

@@ -352,6 +352,7 @@ __device__ __forceinline__ void store_elems(const Vec& s, const TensorRec& t, ui
 
 }  // namespace collage
 #include "step_pipeline.cuh"
+#include "step_direct.cuh"
 namespace collage {
 
 // Sums the per-block partials in a fixed order and writes the EDQ record (Eq. 3).
@@ -486,7 +487,7 @@ static collage_status_t make_scalars(const collage_hyper_t* hyper, uint64_t step
     k->neg_a = dup(s[8] ^ 0x8000u);
     k->lam = dup(s[9]);
     k->eps = dup(s[10]);
-    k->flags = hyper->flags;
+    k->flags = hyper->flags & 7u;          // the kernels know the arithmetic flags only
     {   // float scalars of the register variant: each expression in double, one cast
         const double t = static_cast<double>(step);
         k->f.b1 = static_cast<float>(hyper->beta1);
@@ -597,10 +598,75 @@ static cudaError_t dispatch_step(const StepParams& p, int strategy, bool edq, in
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// ---- small flat tensors: the direct kernel (step_direct.cuh) ---------------------------------
+// Flat tensors up to this many parameters take the direct kernel.  Measured on B200 (Collage-plus with
+// EDQ, steps replayed from a CUDA graph): see the size sweep in profiles/.
+#ifndef COLLAGE_DIRECT_MAX_N
+#define COLLAGE_DIRECT_MAX_N (1ull << 21)
+#endif
+
+template <int STRATEGY, bool EDQ, bool FAST, bool VARIANT>
+static cudaError_t launch_direct(const StepParams& p, int sm_count, cudaStream_t stream, int* grid_out) {
+    auto kernel = adamw_step_direct_kernel<STRATEGY, EDQ, FAST, VARIANT>;
+    static std::atomic<int> per_device[64];
+    int device = 0;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    int blocks_per_sm = per_device[device].load(std::memory_order_acquire);
+    if (blocks_per_sm == 0) {
+        int b = 0;
+        const cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&b, kernel, kDirectThreads, 0);
+        if (e != cudaSuccess) return e;
+        blocks_per_sm = b > 0 ? b : 1;
+        per_device[device].store(blocks_per_sm, std::memory_order_release);
+    }
+    const uint64_t nvec = (p.flat.n + 7) >> 3;
+    uint64_t grid = (nvec + kDirectThreads - 1) / kDirectThreads;
+    const uint64_t resident = static_cast<uint64_t>(sm_count) * blocks_per_sm;
+    if (grid > resident) grid = resident;
+    if (grid > static_cast<uint64_t>(kMaxGrid)) grid = kMaxGrid;
+    *grid_out = static_cast<int>(grid);
+    kernel<<<static_cast<unsigned>(grid), kDirectThreads, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+template <bool FAST, bool VARIANT>
+static cudaError_t dispatch_direct2(const StepParams& p, int strategy, bool edq, int sm_count, cudaStream_t stream,
+                                    int* grid_out) {
+    switch (strategy * 2 + (edq ? 1 : 0)) {
+        case 0: return launch_direct<0, false, FAST, VARIANT>(p, sm_count, stream, grid_out);
+        case 1: return launch_direct<0, true, FAST, VARIANT>(p, sm_count, stream, grid_out);
+        case 2: return launch_direct<1, false, FAST, VARIANT>(p, sm_count, stream, grid_out);
+        case 3: return launch_direct<1, true, FAST, VARIANT>(p, sm_count, stream, grid_out);
+        case 4: return launch_direct<2, false, FAST, VARIANT>(p, sm_count, stream, grid_out);
+        case 5: return launch_direct<2, true, FAST, VARIANT>(p, sm_count, stream, grid_out);
+        default: break;
+    }
+    if constexpr (!VARIANT) {
+        switch (strategy * 2 + (edq ? 1 : 0)) {
+            case 6: return launch_direct<3, false, FAST, false>(p, sm_count, stream, grid_out);
+            case 7: return launch_direct<3, true, FAST, false>(p, sm_count, stream, grid_out);
+            case 8: return launch_direct<4, false, false, false>(p, sm_count, stream, grid_out);
+            case 9: return launch_direct<4, true, false, false>(p, sm_count, stream, grid_out);
+            default: break;
+        }
+    }
+    return cudaErrorInvalidValue;
+}
+
+static cudaError_t dispatch_direct(const StepParams& p, int strategy, bool edq, int sm_count, cudaStream_t stream,
+                                   int* grid_out) {
+    const bool variant = (p.k.flags & (COLLAGE_FLAG_TWOSUM_GROW | COLLAGE_FLAG_DECAY_BY_GROW)) != 0;
+    if (variant)
+        return p.k.fast ? dispatch_direct2<true, true>(p, strategy, edq, sm_count, stream, grid_out)
+                        : dispatch_direct2<false, true>(p, strategy, edq, sm_count, stream, grid_out);
+    return p.k.fast ? dispatch_direct2<true, false>(p, strategy, edq, sm_count, stream, grid_out)
+                    : dispatch_direct2<false, false>(p, strategy, edq, sm_count, stream, grid_out);
+}
+
 // Launches the flat (single tensor) step on device pointers; no-op for n == 0.
 static cudaError_t launch_flat(void* x_hi, void* x_lo, void* m, void* v_hi, void* v_lo, const void* grad, uint64_t n,
                                const StepScalars& k, int strategy, const EdqFinish& fin, int sm_count,
-                               cudaStream_t stream, int* grid_out) {
+                               cudaStream_t stream, int* grid_out, uint32_t kernel_choice = 0) {
     *grid_out = 0;
     if (n == 0) return cudaSuccess;
     StepParams p{};
@@ -622,6 +688,9 @@ static cudaError_t launch_flat(void* x_hi, void* x_lo, void* m, void* v_hi, void
     p.chunk_elems = chunk;
     p.num_chunks = (n + chunk - 1) / chunk;
     p.fin = fin;
+    const bool direct = (kernel_choice & COLLAGE_FLAG_DIRECT_KERNEL) ||
+                        (!(kernel_choice & COLLAGE_FLAG_PIPELINE_KERNEL) && n <= COLLAGE_DIRECT_MAX_N);
+    if (direct) return dispatch_direct(p, strategy, fin.out != nullptr, sm_count, stream, grid_out);
     return dispatch_step<true>(p, strategy, fin.out != nullptr, sm_count, stream, grid_out);
 }
 
@@ -630,8 +699,10 @@ static collage_status_t check_common(const collage_hyper_t* hyper, uint64_t step
     if (step == 0) return COLLAGE_ERR_ARG;
     if (strategy < COLLAGE_BF16 || strategy > COLLAGE_PLUS_FP32_REGISTERS) return COLLAGE_ERR_ARG;
     if (!hyper_in_range(hyper)) return COLLAGE_ERR_ARG;
-    if (hyper->flags & ~(COLLAGE_FLAG_EPS_INSIDE_SQRT | COLLAGE_FLAG_TWOSUM_GROW | COLLAGE_FLAG_DECAY_BY_GROW))
+    if (hyper->flags & ~(COLLAGE_FLAG_EPS_INSIDE_SQRT | COLLAGE_FLAG_TWOSUM_GROW | COLLAGE_FLAG_DECAY_BY_GROW |
+                         COLLAGE_FLAG_PIPELINE_KERNEL | COLLAGE_FLAG_DIRECT_KERNEL))
         return COLLAGE_ERR_ARG;
+    if ((hyper->flags & COLLAGE_FLAG_PIPELINE_KERNEL) && (hyper->flags & COLLAGE_FLAG_DIRECT_KERNEL)) return COLLAGE_ERR_ARG;
     // TwoSum Grow needs a parameter pair (B, C); the Kahan comparator takes neither variant
     if ((hyper->flags & COLLAGE_FLAG_TWOSUM_GROW) && strategy != COLLAGE_LIGHT && strategy != COLLAGE_PLUS)
         return COLLAGE_ERR_ARG;
@@ -790,7 +861,7 @@ collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi,
     const bool edq = hyper->edq_out != nullptr;
     int grid = 0;
     if (launch_flat(x_hi, x_lo, m, v_hi, v_lo, grad, n, k, strategy, make_finish(hyper->workspace, hyper->edq_out, n, false),
-                    dev.sm_count, cs, &grid) != cudaSuccess)
+                    dev.sm_count, cs, &grid, hyper->flags) != cudaSuccess)
         return COLLAGE_ERR_CUDA;
     if (edq && grid == 0) {        // nothing was launched (n == 0): the record still has to say so
         launch_edq_finalize(static_cast<EdqPartial*>(hyper->workspace), 0, 0, static_cast<collage_edq_t*>(hyper->edq_out), cs, false);
@@ -1201,7 +1272,7 @@ collage_status_t collage_adamw_step_host(void* x_hi, void* x_lo, void* m, void* 
         int grid = 0;
         COLLAGE_TRY(launch_flat(dev_array(b, 0), x_lo ? dev_array(b, 1) : nullptr, dev_array(b, 2), dev_array(b, 3),
                                 v_lo ? dev_array(b, 4) : nullptr, dev_array(b, 5), len, k, strategy,
-                                make_finish(partials, edq ? record : nullptr, len, true), dev.sm_count, cs, &grid));
+                                make_finish(partials, edq ? record : nullptr, len, true), dev.sm_count, cs, &grid, h.flags));
         COLLAGE_TRY(cudaEventRecord(c->computed[b], cs));
         COLLAGE_TRY(cudaStreamWaitEvent(c->out, c->computed[b], 0));
         for (int a = 0; a < 5; ++a)

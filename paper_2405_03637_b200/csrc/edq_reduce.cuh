@@ -26,7 +26,7 @@ constexpr int kFinishThreads = 256;
 struct EdqFinishSmem {
     double dot[kFinishThreads / 32], sq[kFinishThreads / 32];
     unsigned long long lost[kFinishThreads / 32];
-    unsigned int is_last;
+    unsigned int is_last, fault;
 };
 
 // Called by EVERY thread of the block (it contains block-wide barriers) once the block's own sums
@@ -50,6 +50,8 @@ __device__ __forceinline__ void edq_publish_and_finish(const EdqFinish& f, EdqFi
     __threadfence();                                        // other blocks' partials, written before their tickets
     double sd = 0.0, sq = 0.0;
     unsigned long long sl = 0;
+    // one thread fetches the fault word while the others fetch the partials (every block's waits are over)
+    if (threadIdx.x == kFinishThreads - 1) sm.fault = fault_word ? *reinterpret_cast<const volatile unsigned int*>(fault_word) : 0u;
     if (threadIdx.x < kFinishThreads) {
         for (unsigned int i = threadIdx.x; i < gridDim.x; i += kFinishThreads) {    // index order per thread
             const double2 a = __ldcg(reinterpret_cast<const double2*>(&f.partials[i]));
@@ -79,7 +81,7 @@ __device__ __forceinline__ void edq_publish_and_finish(const EdqFinish& f, EdqFi
             sumsq += sm.sq[w];
             lost += sm.lost[w];
         }
-        unsigned long long fault = fault_word ? *reinterpret_cast<const volatile unsigned int*>(fault_word) : 0u;
+        unsigned long long fault = sm.fault;
         if (f.accumulate) {
             dot += f.out->dot;
             sumsq += f.out->sumsq;

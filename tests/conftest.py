@@ -37,6 +37,22 @@ def library_under_test_is_the_product_build():
     assert Path(binding.lib()._name) == ROOT / "paper_2405_03637_b200" / "libcollage_b200.so"
 
 
+@pytest.fixture(params=["kernel chosen by size", "pipeline kernel"])
+def step_kernel(request, monkeypatch):
+    """Runs a test twice: as a caller would (small flat tensors take the kernel without staging), and with
+    the bulk-copy pipeline kernel pinned, so that the kernel that streams the large sets sees every edge case."""
+    from paper_2405_03637_b200 import binding
+    if request.param == "pipeline kernel":
+        make = binding.make_hyper
+
+        def pinned(*args, **kwargs):
+            h = make(*args, **kwargs)
+            h.flags |= binding.FLAG_PIPELINE_KERNEL
+            return h
+        monkeypatch.setattr(binding, "make_hyper", pinned)
+    return request.param
+
+
 def bf16_window(e_lo: int, e_hi: int, signs=(0, 1), with_zero=False) -> np.ndarray:
     """All bfloat16 bit patterns whose unbiased exponent is in [e_lo, e_hi] (normal numbers)."""
     out = []

@@ -8,7 +8,7 @@ from gpu_util import EdqBuffers, assert_same_bits, edq_close, oracle_state, orac
 from paper_2405_03637_b200 import binding as B
 from paper_2405_03637_b200 import workloads as W
 
-pytestmark = pytest.mark.gpu
+pytestmark = [pytest.mark.gpu, pytest.mark.usefixtures("step_kernel")]
 KEYS = ("x_hi", "x_lo", "m", "v_hi", "v_lo")
 
 

@@ -19,7 +19,8 @@ def test_bench_line_on_the_reduced_workload():
     j = json.loads(lines[0])
     assert j["metric"] == "collage_adamw_step_params_per_sec" and j["unit"] == "params/s" and j["dtype"] == "bf16"
     assert j["n_gpus"] == 1 and j["steps"] == 4 and j["warmup"] == 3 and j["scaling"] == "weak" and j["data"] == "synthetic"
-    assert j["gpu_launches"] == 8 and j["vs_baseline"] is None and "workload" in j["config"]
+    assert j["gpu_launches"] == 4 and j["vs_baseline"] is None and "workload" in j["config"]      # one launch per step
+    assert j["build_flavor"] == "product" and j["edq_fault"] == 0
     r = j["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["peak"] > 0 and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
     assert 0.9 < r["traffic"] / r["algorithmic"] < 1.1
@@ -30,3 +31,27 @@ def test_bench_line_on_the_reduced_workload():
     assert e["value"] < j["value"]                      # host copies are inside its timed region
     c = j["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] >= 1 and c["value"] > 0 and c["value_one_thread"] > 0
+    assert c["config0_whole"]["value"] > 0
+
+
+def test_sharded_flow_with_two_emulated_ranks_through_the_benchmarks_own_code():
+    # the flow the N-rank run times (one parameter set cut over the ranks, theta stored into every rank's full
+    # copy by the step kernel, EDQ records combined), here with both ranks on this GPU one after the other
+    p = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--sharded-selfcheck", "--layers", "1", "--steps", "2"],
+                       cwd=ROOT, capture_output=True, text=True, timeout=900)
+    assert p.returncode == 0, p.stderr[-2000:]
+    j = json.loads([l for l in p.stdout.splitlines() if l.startswith("{")][-1])["sharded_selfcheck"]
+    assert j["ok"] and j["theta_copies_bitwise_equal_to_unsharded"] and j["edq_max_relative_difference"] <= 1e-5
+    assert j["theta_bytes_sent_per_rank_per_step"] == j["params_total"]          # 2 B x half of the parameters x 1 peer
+
+
+@pytest.mark.parametrize("config", [0, 1, 2])
+def test_other_configurations_print_contract_lines(config):
+    p = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--config", str(config)], cwd=ROOT, capture_output=True,
+                       text=True, timeout=900)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [json.loads(l) for l in p.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == {0: 3, 1: 1, 2: 2}[config]
+    for j in lines:
+        assert j["unit"] == "params/s" and j["value"] > 0 and j["gpu_launches_per_step"] == 1
+        assert j["roofline"]["bound"] == "hbm" and 0 < j["roofline"]["frac"] < 1.3

@@ -210,7 +210,7 @@ def test_stress_set_collage_plus_against_plain_bf16():
 
 
 @pytest.mark.parametrize("strategy", [1, 2])
-def test_size_sweep_powers_of_four(strategy):
+def test_size_sweep_powers_of_four(strategy, step_kernel):
     # config 4: flat tensors of 4^6 ... 4^12 parameters, two steps each, every array and EDQ
     dev = torch.device("cuda")
     hyp = W.HYPERS

@@ -10,7 +10,7 @@ from gpu_util import assert_same_bits
 from paper_2405_03637_b200 import binding as B
 from paper_2405_03637_b200 import workloads as W
 
-pytestmark = pytest.mark.gpu
+pytestmark = [pytest.mark.gpu, pytest.mark.usefixtures("step_kernel")]
 CASES = [(0, 0), (1, 0), (2, 0), (3, 0), (1, 2), (2, 2), (2, 4), (2, 7), (0, 4), (0, 1), (2, 1), (3, 1)]
 
 

@@ -8,7 +8,7 @@ from gpu_util import EdqBuffers, Guarded, assert_same_bits, edq_close, oracle_st
 from paper_2405_03637_b200 import binding as B
 from paper_2405_03637_b200 import workloads as W
 
-pytestmark = pytest.mark.gpu
+pytestmark = [pytest.mark.gpu, pytest.mark.usefixtures("step_kernel")]
 
 KEYS = ("x_hi", "x_lo", "m", "v_hi", "v_lo")
 
@@ -213,7 +213,7 @@ def test_host_resident_state_is_staged_with_identical_results(strategy):
         for k in KEYS:
             if st[k] is not None:
                 assert_same_bits(W.bits(host[k]), st[k], f"host step {t} {k}")
-        got = B.Edq.from_buffer_copy(bytes(rec)[:40])
+        got = B.Edq.from_buffer_copy(bytes(rec)[:B.EDQ_RECORD_BYTES])
         edq_close(dict(dot=got.dot, sumsq=got.sumsq, edq=got.edq, lost=int(got.lost)), want)
         assert int(got.n) == n
     with pytest.raises(B.CollageError) as err:
