@@ -281,9 +281,9 @@ def run_sharded_children(args, world):
     if args.lib:
         cmd += ["--lib", args.lib]
     try:
-        proc = subprocess.run(cmd, capture_output=True, text=True, timeout=900, env=env, cwd=str(ROOT))
+        proc = subprocess.run(cmd, capture_output=True, text=True, timeout=420, env=env, cwd=str(ROOT))
     except subprocess.TimeoutExpired:
-        return {"unavailable": "the sharded leg did not finish within 900 s"}
+        return {"unavailable": "the sharded leg did not finish within 420 s"}
     for line in reversed(proc.stdout.splitlines()):
         if line.startswith("{") and '"sharded_step"' in line:
             return json.loads(line)["sharded_step"]
@@ -386,6 +386,7 @@ def run_sharded_only(args):
             "from inside the step kernel; {dot, sumsq, lost} all-reduced (NCCL)", "gpu_launches": args.steps,
         }
         stepper.close()
+        del stepper, shard, copies, flats                            # peers' mappings are released before anyone exits
     except Exception as exc:                                         # noqa: BLE001 - reported, never fatal for the caller
         result = {"unavailable": f"{type(exc).__name__}: {str(exc)[:300]}"}
     finally:
