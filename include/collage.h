@@ -192,7 +192,7 @@ collage_status_t collage_adamw_step(void* x_hi, void* x_lo, void* m, void* v_hi,
  * EDQ (hyper->edq_out / workspace as for collage_adamw_step) measures the float update against the
  * change of the stored parameter: the master weight for D, the bfloat16 parameter for D^-MW.
  * HBM traffic 28 B/param (D) or 22 B/param (D^-MW) against 22 B/param of Collage-plus.
- * Only COLLAGE_FLAG_EPS_INSIDE_SQRT is accepted in hyper->flags.
+ * Of the arithmetic flags only COLLAGE_FLAG_EPS_INSIDE_SQRT is accepted in hyper->flags.
  * Errors: ERR_NULL, ERR_ARG (step 0, hyper range, flags, float arrays not 4-byte aligned),
  * ERR_ALIAS, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA. */
 collage_status_t collage_adamw_step_fp32(void* theta, void* master, void* m, void* v, const void* grad,

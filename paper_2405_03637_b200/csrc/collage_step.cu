@@ -752,7 +752,8 @@ struct collage_plan {
     int num_given = 0;                   // length of the caller's array
     uint64_t* d_replica_bases = nullptr; // [num_replicas][num_tensors] (non-empty tensors only)
     int num_replicas = 0;
-    std::vector<ByteRange> ranges;       // byte ranges of every array of the plan, sorted by address (overlap checks)
+    std::vector<ByteRange> ranges;       // byte ranges of every array of the plan and of its replicas, sorted by address (overlap checks)
+    std::vector<ByteRange> own_ranges;   // the same without the replicas
     std::vector<collage_tensor_t> given; // the caller's array, as given
     uint64_t num_chunks = 0;
     uint64_t num_elements = 0;
@@ -923,6 +924,7 @@ collage_status_t collage_plan_create(const collage_tensor_t* tensors, int num, u
     collage_plan* plan = new collage_plan;
     plan->num_given = num;
     plan->ranges = ranges;
+    plan->own_ranges = ranges;
     plan->given.assign(tensors, tensors + num);
     plan->num_chunks = chunks.size();
     plan->num_elements = total;
@@ -1010,7 +1012,7 @@ collage_status_t collage_plan_set_replicas(collage_plan_t* plan, const void* con
     if (num_replicas > 0 && !replicas) return COLLAGE_ERR_NULL;
     if (!plan_on_current_device(plan)) return COLLAGE_ERR_ARG;
     std::vector<uint64_t> bases;
-    std::vector<ByteRange> ranges = plan->ranges;
+    std::vector<ByteRange> ranges = plan->own_ranges;
     for (int r = 0; r < num_replicas; ++r) {
         for (int i = 0; i < plan->num_given; ++i) {
             const collage_tensor_t& t = plan->given[i];
@@ -1036,6 +1038,7 @@ collage_status_t collage_plan_set_replicas(collage_plan_t* plan, const void* con
     cudaFree(plan->d_replica_bases);
     plan->d_replica_bases = d;
     plan->num_replicas = bases.empty() ? 0 : num_replicas;
+    plan->ranges = ranges;                 // sorted by any_overlap: later calls check their workspace against the replicas too
     return COLLAGE_OK;
 }
 

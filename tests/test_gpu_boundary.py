@@ -149,6 +149,14 @@ def test_record_and_workspace_may_not_overlap_a_plan():
     with pytest.raises(B.CollageError) as err:                       # the record inside the workspace
         B.adamw_step_multi(plan, B.make_hyper(**hyp, edq_out=e.ws[256:320], workspace=e.ws), 1, B.LIGHT)
     assert err.value.status == B.ERR_ALIAS
+    # a registered replica of theta counts as an array of the plan
+    rep = torch.zeros(n * 2 + 64, dtype=torch.uint8, device="cuda")
+    B.plan_set_replicas(plan, [[rep[:n * 2].view(torch.bfloat16)]])
+    with pytest.raises(B.CollageError) as err:
+        B.adamw_step_multi(plan, B.make_hyper(**hyp, edq_out=rep[1024:1088], workspace=e.ws), 1, B.LIGHT)
+    assert err.value.status == B.ERR_ALIAS
+    B.plan_set_replicas(plan, [])
+    B.adamw_step_multi(plan, B.make_hyper(**hyp, edq_out=rep[1024:1088], workspace=e.ws), 1, B.LIGHT)    # no longer a replica
     per = torch.zeros(B.EDQ_RECORD_BYTES, dtype=torch.uint8, device="cuda")
     cws = torch.empty(B.plan_workspace_bytes(plan), dtype=torch.uint8, device="cuda")
     B.adamw_step_multi_per_tensor(plan, B.make_hyper(**hyp), 2, B.LIGHT, per, 1, cws)
@@ -158,6 +166,22 @@ def test_record_and_workspace_may_not_overlap_a_plan():
     torch.cuda.synchronize()
     B.plan_destroy(plan)
     B.plan_destroy(plan2)
+
+
+def test_empty_inputs_still_write_their_record():
+    # n == 0 and an empty plan launch no step kernel; the record must still say "nothing": zeros, not stale data
+    e = EdqBuffers()
+    e.out.fill_(0xAB)
+    z = torch.zeros(8, dtype=torch.bfloat16, device="cuda")
+    B.adamw_step(z, z.clone(), z.clone(), z.clone(), z.clone(), z.clone(), 0, e.hyper(W.HYPERS), 1, B.PLUS)
+    torch.cuda.synchronize()
+    assert e.read() == dict(dot=0.0, sumsq=0.0, edq=0.0, n=0, lost=0, fault=0)
+    e.out.fill_(0xAB)
+    plan = B.plan_create([(z, z.clone(), z.clone(), z.clone(), z.clone(), z.clone(), 0)])
+    B.adamw_step_multi(plan, e.hyper(W.HYPERS), 1, B.PLUS)
+    torch.cuda.synchronize()
+    assert e.read() == dict(dot=0.0, sumsq=0.0, edq=0.0, n=0, lost=0, fault=0)
+    B.plan_destroy(plan)
 
 
 def test_build_flavor_of_the_library_under_test_is_the_product():
