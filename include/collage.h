@@ -85,13 +85,18 @@ typedef enum {
  *   Adam part (-a) (*) r.  A, B, C.  EDQ then measures against d + update. */
 #define COLLAGE_FLAG_TWOSUM_GROW 2u
 #define COLLAGE_FLAG_DECAY_BY_GROW 4u
-/* Which kernel steps a flat tensor (collage_adamw_step, collage_adamw_step_host).  By default the size
- * decides: up to 2^21 parameters a kernel without staging, one 8-parameter vector per thread straight
- * from global memory (shortest latency); above, the bulk-copy pipeline that streams at HBM bandwidth.
- * Both compute the same bits.  These flags pin the choice (tests and measurements); setting both is
- * ERR_ARG; entry points without such a choice ignore them. */
+/* Which kernel runs the step.  By default the size decides: a flat tensor of up to 2^21 parameters takes
+ * a kernel without staging, one 8-parameter vector per thread straight from global memory (shortest
+ * latency); above that, and for every multi-tensor plan, the bulk-copy pipeline streams at HBM bandwidth
+ * in three stages of 4096-element tiles (6144 for COLLAGE_BF16); a COLLAGE_PLUS step over 2^27 parameters or
+ * more uses two stages of 8192-element tiles (1-2 % faster there; in a plan only if chunk_elems is a
+ * multiple of 8192, as the default is).  All of them compute the same bits.  These flags pin the choice
+ * (tests and measurements): PIPELINE_KERNEL = the three-stage pipeline whatever the size, DIRECT_KERNEL =
+ * the kernel without staging (flat entry points only), LARGE_TILES = the two-stage pipeline (COLLAGE_PLUS
+ * without variant flags only).  More than one of them is ERR_ARG; where a flag does not apply it is ignored. */
 #define COLLAGE_FLAG_PIPELINE_KERNEL 8u
 #define COLLAGE_FLAG_DIRECT_KERNEL 16u
+#define COLLAGE_FLAG_LARGE_TILES 32u
 
 /* Hyper-parameters of one step (Algorithm 2 line 1).  HOST struct.
  * Valid ranges: lr, eps, weight_decay >= 0 and finite; 0 <= beta1, beta2 < 1. */

@@ -14,7 +14,7 @@ _LIB_PATH = Path(__file__).resolve().parent / "libcollage_b200.so"      # the in
 OK, ERR_NULL, ERR_ARG, ERR_ALIAS, ERR_ARCH, ERR_CUDA, ERR_WORKSPACE, ERR_LIMIT = range(8)
 BF16, LIGHT, PLUS, KAHAN, PLUS_FP32_REGISTERS = 0, 1, 2, 3, 4
 FLAG_EPS_INSIDE_SQRT, FLAG_TWOSUM_GROW, FLAG_DECAY_BY_GROW = 1, 2, 4
-FLAG_PIPELINE_KERNEL, FLAG_DIRECT_KERNEL = 8, 16
+FLAG_PIPELINE_KERNEL, FLAG_DIRECT_KERNEL, FLAG_LARGE_TILES = 8, 16, 32
 OP_ADD, OP_SUB, OP_MUL, OP_DIV, OP_SQRT, OP_FMA = range(6)
 SCALAR_NAMES = ("b1", "c1", "b2", "c2", "b2h", "b2l", "bc1", "bc2", "a", "lam", "eps")
 

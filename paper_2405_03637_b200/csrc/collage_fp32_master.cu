@@ -340,7 +340,7 @@ extern "C" collage_status_t collage_adamw_step_fp32(void* theta, void* master, v
                                                     void* stream) {
     if (!hyper) return COLLAGE_ERR_NULL;
     if (step == 0 || !hyper_in_range(hyper)) return COLLAGE_ERR_ARG;
-    if (hyper->flags & ~(COLLAGE_FLAG_EPS_INSIDE_SQRT | COLLAGE_FLAG_PIPELINE_KERNEL | COLLAGE_FLAG_DIRECT_KERNEL))
+    if (hyper->flags & ~(COLLAGE_FLAG_EPS_INSIDE_SQRT | COLLAGE_FLAG_PIPELINE_KERNEL | COLLAGE_FLAG_DIRECT_KERNEL | COLLAGE_FLAG_LARGE_TILES))
         return COLLAGE_ERR_ARG;                               // the kernel-choice flags mean nothing here and are ignored
     if (hyper->edq_out) {
         if (!hyper->workspace || hyper->workspace_bytes < kWorkspaceBytes ||

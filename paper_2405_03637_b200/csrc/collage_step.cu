@@ -69,9 +69,19 @@ constexpr PipeGeometry pipe_geometry(int strategy) {
                ? PipeGeometry{COLLAGE_PIPE_CONSUMERS_B, COLLAGE_PIPE_VPT_B, COLLAGE_PIPE_STAGES_B}
                : PipeGeometry{COLLAGE_PIPE_CONSUMERS, COLLAGE_PIPE_VPT, COLLAGE_PIPE_STAGES};
 }
+// Option C on LARGE parameter sets: two stages of 8192-element tiles (two vectors per consumer thread), the
+// same shared memory within 33 %.  Fewer, larger copies in flight stream 1-2 % faster from 2^28 parameters on
+// (measured, interleaved, on one device: 4.221 against 4.305 ms on 1.27 G parameters, 0.900 against 0.913 ms
+// on 2^28), are equal at 2^25..2^27 and slower below (a tensor of a few million parameters has too few tiles
+// per block for tiles twice as long).
+#ifndef COLLAGE_LARGE_TILE_MIN_N
+#define COLLAGE_LARGE_TILE_MIN_N (1ull << 27)
+#endif
+constexpr PipeGeometry kLargeGeometry = {512, 2, 2};
 // elements per tile
-constexpr uint32_t pipe_tile(int strategy) {
-    return static_cast<uint32_t>(pipe_geometry(strategy).consumers) * 8u * static_cast<uint32_t>(pipe_geometry(strategy).vpt);
+constexpr uint32_t pipe_tile(int strategy, bool large = false) {
+    return large ? static_cast<uint32_t>(kLargeGeometry.consumers) * 8u * static_cast<uint32_t>(kLargeGeometry.vpt)
+                 : static_cast<uint32_t>(pipe_geometry(strategy).consumers) * 8u * static_cast<uint32_t>(pipe_geometry(strategy).vpt);
 }
 
 struct TensorRec {
@@ -509,10 +519,11 @@ static collage_status_t make_scalars(const collage_hyper_t* hyper, uint64_t step
     return COLLAGE_OK;
 }
 
-template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, bool PER_CHUNK = false, bool VARIANT = false>
+template <int STRATEGY, bool EDQ, bool FLAT, bool FAST, bool PER_CHUNK = false, bool VARIANT = false, bool LARGE = false>
 static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t stream, int* grid_out) {
-    constexpr int CONSUMERS = pipe_geometry(STRATEGY).consumers;
-    constexpr int VPT = pipe_geometry(STRATEGY).vpt, STAGES = pipe_geometry(STRATEGY).stages;
+    constexpr PipeGeometry G = LARGE ? kLargeGeometry : pipe_geometry(STRATEGY);
+    constexpr int CONSUMERS = G.consumers;
+    constexpr int VPT = G.vpt, STAGES = G.stages;
     auto kernel = adamw_step_pipeline_kernel<STRATEGY, EDQ, FLAT, FAST, CONSUMERS, VPT, STAGES, PER_CHUNK, VARIANT>;
     constexpr size_t smem = sizeof(PipeSmem<CONSUMERS, VPT, STAGES, STRATEGY>) + 128;
     constexpr int threads = CONSUMERS + 32;
@@ -541,7 +552,10 @@ static cudaError_t launch_step(const StepParams& p, int sm_count, cudaStream_t s
 
 template <bool FLAT, bool FAST>
 static cudaError_t dispatch_step2(const StepParams& p, int strategy, bool edq, int sm_count, cudaStream_t stream,
-                                  int* grid_out) {
+                                  int* grid_out, bool large) {
+    if (large && strategy == 2)
+        return edq ? launch_step<2, true, FLAT, FAST, false, false, true>(p, sm_count, stream, grid_out)
+                   : launch_step<2, false, FLAT, FAST, false, false, true>(p, sm_count, stream, grid_out);
     switch (strategy * 2 + (edq ? 1 : 0)) {
         case 0: return launch_step<0, false, FLAT, FAST>(p, sm_count, stream, grid_out);
         case 1: return launch_step<0, true, FLAT, FAST>(p, sm_count, stream, grid_out);
@@ -586,14 +600,21 @@ static cudaError_t dispatch_variant(const StepParams& p, int strategy, bool edq,
     }
 }
 
+// Does a Collage-plus step over `n` parameters take the large tiles?  `choice` = the kernel-choice flags.
+static bool takes_large_tiles(int strategy, uint32_t arithmetic_flags, uint32_t choice, uint64_t n) {
+    if (strategy != COLLAGE_PLUS || (arithmetic_flags & (COLLAGE_FLAG_TWOSUM_GROW | COLLAGE_FLAG_DECAY_BY_GROW))) return false;
+    if (choice & COLLAGE_FLAG_LARGE_TILES) return true;
+    return !(choice & COLLAGE_FLAG_PIPELINE_KERNEL) && n >= COLLAGE_LARGE_TILE_MIN_N;
+}
+
 template <bool FLAT>
 static cudaError_t dispatch_step(const StepParams& p, int strategy, bool edq, int sm_count, cudaStream_t stream,
-                                 int* grid_out) {
+                                 int* grid_out, bool large = false) {
     if (p.k.flags & (COLLAGE_FLAG_TWOSUM_GROW | COLLAGE_FLAG_DECAY_BY_GROW))
         return p.k.fast ? dispatch_variant<FLAT, true>(p, strategy, edq, sm_count, stream, grid_out)
                         : dispatch_variant<FLAT, false>(p, strategy, edq, sm_count, stream, grid_out);
-    return p.k.fast ? dispatch_step2<FLAT, true>(p, strategy, edq, sm_count, stream, grid_out)
-                    : dispatch_step2<FLAT, false>(p, strategy, edq, sm_count, stream, grid_out);
+    return p.k.fast ? dispatch_step2<FLAT, true>(p, strategy, edq, sm_count, stream, grid_out, large)
+                    : dispatch_step2<FLAT, false>(p, strategy, edq, sm_count, stream, grid_out, large);
 }
 
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -682,16 +703,17 @@ static cudaError_t launch_flat(void* x_hi, void* x_lo, void* m, void* v_hi, void
                      aligned16(grad);
     // four tiles per chunk when there is plenty of work, one tile per chunk when the tensor is small,
     // so that every SM still gets a share
-    const uint32_t tile = pipe_tile(strategy);
+    const bool large = takes_large_tiles(strategy, k.flags, kernel_choice, n);
+    const uint32_t tile = pipe_tile(strategy, large);
     uint32_t chunk = 4 * tile;
     if ((n + chunk - 1) / chunk < 4ull * static_cast<uint64_t>(sm_count)) chunk = tile;
     p.chunk_elems = chunk;
     p.num_chunks = (n + chunk - 1) / chunk;
     p.fin = fin;
     const bool direct = (kernel_choice & COLLAGE_FLAG_DIRECT_KERNEL) ||
-                        (!(kernel_choice & COLLAGE_FLAG_PIPELINE_KERNEL) && n <= COLLAGE_DIRECT_MAX_N);
+                        (!(kernel_choice & (COLLAGE_FLAG_PIPELINE_KERNEL | COLLAGE_FLAG_LARGE_TILES)) && n <= COLLAGE_DIRECT_MAX_N);
     if (direct) return dispatch_direct(p, strategy, fin.out != nullptr, sm_count, stream, grid_out);
-    return dispatch_step<true>(p, strategy, fin.out != nullptr, sm_count, stream, grid_out);
+    return dispatch_step<true>(p, strategy, fin.out != nullptr, sm_count, stream, grid_out, large);
 }
 
 static collage_status_t check_common(const collage_hyper_t* hyper, uint64_t step, int strategy) {
@@ -700,9 +722,12 @@ static collage_status_t check_common(const collage_hyper_t* hyper, uint64_t step
     if (strategy < COLLAGE_BF16 || strategy > COLLAGE_PLUS_FP32_REGISTERS) return COLLAGE_ERR_ARG;
     if (!hyper_in_range(hyper)) return COLLAGE_ERR_ARG;
     if (hyper->flags & ~(COLLAGE_FLAG_EPS_INSIDE_SQRT | COLLAGE_FLAG_TWOSUM_GROW | COLLAGE_FLAG_DECAY_BY_GROW |
-                         COLLAGE_FLAG_PIPELINE_KERNEL | COLLAGE_FLAG_DIRECT_KERNEL))
+                         COLLAGE_FLAG_PIPELINE_KERNEL | COLLAGE_FLAG_DIRECT_KERNEL | COLLAGE_FLAG_LARGE_TILES))
         return COLLAGE_ERR_ARG;
-    if ((hyper->flags & COLLAGE_FLAG_PIPELINE_KERNEL) && (hyper->flags & COLLAGE_FLAG_DIRECT_KERNEL)) return COLLAGE_ERR_ARG;
+    {   // at most one kernel choice
+        const uint32_t choice = hyper->flags & (COLLAGE_FLAG_PIPELINE_KERNEL | COLLAGE_FLAG_DIRECT_KERNEL | COLLAGE_FLAG_LARGE_TILES);
+        if (choice & (choice - 1)) return COLLAGE_ERR_ARG;
+    }
     // TwoSum Grow needs a parameter pair (B, C); the Kahan comparator takes neither variant
     if ((hyper->flags & COLLAGE_FLAG_TWOSUM_GROW) && strategy != COLLAGE_LIGHT && strategy != COLLAGE_PLUS)
         return COLLAGE_ERR_ARG;
@@ -997,7 +1022,10 @@ collage_status_t collage_adamw_step_multi(const collage_plan_t* plan, const coll
     p.num_plan_tensors = plan->num_tensors;
     int grid = 0;
     if (plan->num_chunks > 0) {
-        if (dispatch_step<false>(p, strategy, edq, dev.sm_count, cs, &grid) != cudaSuccess) return COLLAGE_ERR_CUDA;
+        // large tiles need chunks that are whole numbers of them (the default chunk is three)
+        const bool large = plan->chunk_elems % pipe_tile(COLLAGE_PLUS, true) == 0 &&
+                           takes_large_tiles(strategy, p.k.flags, hyper->flags, plan->num_elements);
+        if (dispatch_step<false>(p, strategy, edq, dev.sm_count, cs, &grid, large) != cudaSuccess) return COLLAGE_ERR_CUDA;
     }
     if (edq && grid == 0) {        // an empty plan: the record still has to say so
         launch_edq_finalize(p.fin.partials, 0, 0, p.fin.out, cs, false);

@@ -37,17 +37,20 @@ def library_under_test_is_the_product_build():
     assert Path(binding.lib()._name) == ROOT / "paper_2405_03637_b200" / "libcollage_b200.so"
 
 
-@pytest.fixture(params=["kernel chosen by size", "pipeline kernel"])
+@pytest.fixture(params=["kernel chosen by size", "pipeline kernel", "large-tile pipeline"])
 def step_kernel(request, monkeypatch):
-    """Runs a test twice: as a caller would (small flat tensors take the kernel without staging), and with
-    the bulk-copy pipeline kernel pinned, so that the kernel that streams the large sets sees every edge case."""
+    """Runs a test three times: as a caller would (small flat tensors take the kernel without staging), with
+    the three-stage bulk-copy pipeline pinned, and with the two-stage large-tile pipeline pinned (it applies to
+    Collage-plus; other options then run as chosen by size), so that the kernels that stream the large sets
+    see every edge case too."""
     from paper_2405_03637_b200 import binding
-    if request.param == "pipeline kernel":
+    pin = {"pipeline kernel": binding.FLAG_PIPELINE_KERNEL, "large-tile pipeline": binding.FLAG_LARGE_TILES}.get(request.param)
+    if pin:
         make = binding.make_hyper
 
         def pinned(*args, **kwargs):
             h = make(*args, **kwargs)
-            h.flags |= binding.FLAG_PIPELINE_KERNEL
+            h.flags |= pin
             return h
         monkeypatch.setattr(binding, "make_hyper", pinned)
     return request.param

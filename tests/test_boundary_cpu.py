@@ -82,9 +82,10 @@ def test_argument_errors_are_reported_before_any_cuda_call(L):
         kw = dict(lr=1e-4, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.1)
         kw.update(bad)
         assert call(hyper=B.make_hyper(**kw)) == B.ERR_ARG
-    assert call(hyper=B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1, flags=32)) == B.ERR_ARG
+    assert call(hyper=B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1, flags=64)) == B.ERR_ARG
     both = B.FLAG_PIPELINE_KERNEL | B.FLAG_DIRECT_KERNEL                      # contradictory kernel choice
     assert call(hyper=B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1, flags=both)) == B.ERR_ARG
+    assert call(hyper=B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1, flags=B.FLAG_LARGE_TILES | B.FLAG_PIPELINE_KERNEL)) == B.ERR_ARG
     # variant flags only where they mean something
     assert call(hyper=B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1, flags=B.FLAG_TWOSUM_GROW)) == B.ERR_ARG      # option A
     kahan_bad = B.make_hyper(1e-4, 0.9, 0.999, 1e-8, 0.1, flags=B.FLAG_DECAY_BY_GROW)

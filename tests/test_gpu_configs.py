@@ -51,7 +51,9 @@ def test_llama7b_full_size_launch_sampled_parity():
     assert total >= 2 ** 28
     hyp = W.HYPERS
     for t in (1, 2):
-        B.adamw_step_multi(plan, e.hyper(hyp), t, B.PLUS)
+        # step 1 as bench.py launches it (at this size: the two-stage pipeline with 8192-element tiles), step 2
+        # with the three-stage pipeline pinned, so that both are checked at full size
+        B.adamw_step_multi(plan, e.hyper(hyp, flags=0 if t == 1 else B.FLAG_PIPELINE_KERNEL), t, B.PLUS)
         torch.cuda.synchronize()
         for i, wins, st, g in samples:
             oracle_step(st, g, t, 2, hyp)
@@ -289,8 +291,8 @@ def test_one_tensor_longer_than_2_to_32_elements(api):
     e = EdqBuffers()
     plan = B.plan_create([(x, xl, m, v, vl, g, n)]) if api == "multi" else None
     for t in (1, 2):
-        if api == "multi":
-            B.adamw_step_multi(plan, e.hyper(W.HYPERS), t, B.PLUS)
+        if api == "multi":      # the plan with the three-stage pipeline pinned, the flat call as chosen by size (large tiles)
+            B.adamw_step_multi(plan, e.hyper(W.HYPERS, flags=B.FLAG_PIPELINE_KERNEL), t, B.PLUS)
         else:
             B.adamw_step(x, xl, m, v, vl, g, n, e.hyper(W.HYPERS), t, B.PLUS)
         torch.cuda.synchronize()
