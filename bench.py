@@ -39,9 +39,9 @@ STRATEGY_NAME = {0: "plain_bf16", 1: "collage_light", 2: "collage_plus"}
 STRATEGY = 2                                  # Collage-plus
 WORKLOAD = "llama7b_shaped_291_tensors_collage_plus_with_edq"
 # DRAM bytes per parameter of the step kernel from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum = 3.146 GB + 2.567 GB on the 262,148,096-parameter case, summary under
+# dram__bytes_write.sum = 3.146 GB + 2.565 GB on the 262,148,096-parameter case, summary under
 # profiles/); every byte is touched once, so traffic scales with the parameter count.
-NCU_TRAFFIC_BYTES_PER_PARAM = (3.146235e9 + 2.567421e9) / 262_148_096
+NCU_TRAFFIC_BYTES_PER_PARAM = (3.146280e9 + 2.564761e9) / 262_148_096
 
 
 def host_threads():
@@ -189,11 +189,13 @@ def run_collage(args):
         per = torch.zeros(len(rows) * B.EDQ_RECORD_BYTES, dtype=torch.uint8, device=device)
         cws = torch.empty(B.plan_workspace_bytes(plan), dtype=torch.uint8, device=device)
 
+    pin = {"auto": 0, "pipeline": B.FLAG_PIPELINE_KERNEL, "large": B.FLAG_LARGE_TILES}[args.pin_kernel]
+
     def step(t):
         if args.per_tensor:
             B.adamw_step_multi_per_tensor(plan, B.make_hyper(**hyp, edq_out=edq_dev), t, STRATEGY, per, len(rows), cws, stream)
         else:
-            B.adamw_step_multi(plan, B.make_hyper(**hyp, edq_out=edq_dev, workspace=ws), t, STRATEGY, stream)
+            B.adamw_step_multi(plan, B.make_hyper(**hyp, flags=pin, edq_out=edq_dev, workspace=ws), t, STRATEGY, stream)
         if use_dist:                                    # EDQ is global: sum the partial sums over ranks
             dist.all_reduce(edq_sums)
             dist.all_reduce(edq_lost)
@@ -243,7 +245,10 @@ def run_collage(args):
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": NCU_TRAFFIC_BYTES_PER_PARAM * n / 1e9, "traffic_unit": "GB per launch (ncu, scaled by parameters)",
                      "algorithmic": n * BYTES_PER_PARAM[STRATEGY] / 1e9, "peak_source": peak_src, "frac_of_nominal_8TBps": achieved / 8000.0,
-                     "kernel": "adamw_step_pipeline_kernel<C, EDQ, multi-tensor>", "kernel_ms": kernel_ms},
+                     "kernel": "adamw_step_pipeline_kernel<C, EDQ, multi-tensor, " +
+                               ("2 stages x 8192-element tiles>" if (args.pin_kernel == "large" or (args.pin_kernel == "auto" and n >= 1 << 27
+                                                                     and (args.chunk_elems or 24576) % 8192 == 0))
+                                else "3 stages x 4096-element tiles>"), "kernel_ms": kernel_ms},
         "clocks": clocks.summary(),
         "edq": edq["edq"], "edq_fault": edq["fault"],
     }
@@ -890,6 +895,8 @@ def main():
                     help="synthetic configuration to time (3 = the LLaMA-7B-shaped headline; 4 = the size sweep)")
     ap.add_argument("--primitive-sweep", action="store_true", help="time the batched primitives and the stand-alone EDQ")
     ap.add_argument("--lib", default=None, help="another build of the library (build.py --out), e.g. the data-movement-only build")
+    ap.add_argument("--pin-kernel", default="auto", choices=["auto", "pipeline", "large"],
+                    help="headline step: kernel as chosen by size, or pin the three-stage / the large-tile pipeline (A/B runs)")
     ap.add_argument("--no-sharded", action="store_true", help="N > 1: skip the sharded-step record")
     ap.add_argument("--sharded-only", action="store_true", help="(internal) run only the sharded step, under torchrun")
     ap.add_argument("--sharded-selfcheck", action="store_true", help="the sharded flow with two emulated ranks on one GPU")
