@@ -327,9 +327,18 @@ def run_sharded_only(args):
     from paper_2405_03637_b200 import workloads as W
     B = load_binding(args)
     rank, local_rank, world = int(os.environ["RANK"]), int(os.environ["LOCAL_RANK"]), int(os.environ["WORLD_SIZE"])
+    if args.sharded_one_device:
+        # test mode for a box with one GPU: every rank is a process of its own on device 0, so the handle
+        # exchange, the mapping of another process's memory and the stores into it are the real ones; only
+        # the sums travel over gloo (NCCL does not take two ranks on one device).  The ranks' kernels never
+        # wait on one another, so sharing a device is safe.
+        local_rank = 0
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
-    dist.init_process_group("nccl", device_id=device)
+    if args.sharded_backend == "gloo":
+        dist.init_process_group("gloo")
+    else:
+        dist.init_process_group("nccl", device_id=device)
     result = None
     try:
         sizes = [n for _, n in W.llama7b_shapes(args.layers)]
@@ -345,7 +354,8 @@ def run_sharded_only(args):
             if r == rank:
                 flats[r] = mine_flat
             else:
-                B.enable_peer_access(peer_device)
+                if peer_device != local_rank:
+                    B.enable_peer_access(peer_device)
                 flats[r] = rebuild_cuda_tensor(*ipc)
         copies = [theta_views(flats[r], sizes) for r in range(world)]
         alloc = lambda n: torch.zeros(n, dtype=torch.bfloat16, device=device)
@@ -388,7 +398,8 @@ def run_sharded_only(args):
             "expected_ms": {"hbm": hbm_ms, "nvlink_at_770_gbs": link_ms, "bound": max(hbm_ms, link_ms)},
             "frac_of_bound": max(hbm_ms, link_ms) / ms, "copies_agree": len(set(sums)) == 1,
             "edq": edq["edq"], "edq_fault": edq["fault"], "exchange": "plain stores into CUDA-IPC mapped peer memory "
-            "from inside the step kernel; {dot, sumsq, lost} all-reduced (NCCL)", "gpu_launches": args.steps,
+            "from inside the step kernel; {dot, sumsq, lost} all-reduced (" + args.sharded_backend + ")",
+            "gpu_launches": args.steps,
         }
         stepper.close()
         del stepper, shard, copies, flats                            # peers' mappings are released before anyone exits
@@ -900,6 +911,9 @@ def main():
     ap.add_argument("--no-sharded", action="store_true", help="N > 1: skip the sharded-step record")
     ap.add_argument("--sharded-only", action="store_true", help="(internal) run only the sharded step, under torchrun")
     ap.add_argument("--sharded-selfcheck", action="store_true", help="the sharded flow with two emulated ranks on one GPU")
+    ap.add_argument("--sharded-backend", default="nccl", choices=["nccl", "gloo"], help="--sharded-only: how the EDQ sums travel")
+    ap.add_argument("--sharded-one-device", action="store_true",
+                    help="--sharded-only test mode: all ranks are separate processes on device 0 (use with --sharded-backend gloo)")
     args = ap.parse_args()
     if args.sharded_only:
         run_sharded_only(args)

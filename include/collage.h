@@ -225,7 +225,7 @@ collage_status_t collage_adamw_step_host(void* x_hi, void* x_lo, void* m, void* 
  * collage_plan_create copies the HOST array `tensors[num]` and builds the device table
  * (this call allocates and synchronises; do it once, outside the step loop).  chunk_elems is
  * the work unit handed to a thread block, a multiple of 2048; 0 picks the default (24576;
- * multiples of 12288 keep every tile whole for all three precision options).
+ * multiples of 24576 keep every tile whole for every precision option and tile size).
  * Tensors with n == 0 are skipped.  The plan records which pointers were NULL; a step whose
  * strategy needs a missing component fails with ERR_NULL.  EDQ is over all tensors (Eq. 3
  * with theta the concatenation).

@@ -140,10 +140,17 @@ class CudaStepper:
                            self.shard.strategy, stream)
 
     def allreduce(self, dist):
-        """Sum the EDQ partial sums over ranks on the device (no host synchronisation)."""
+        """Sum the EDQ partial sums over ranks: on the device over NCCL (no host synchronisation), through
+        host copies when the process group is gloo (CPU tests of the flow)."""
         if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
-            dist.all_reduce(self.sums)
-            dist.all_reduce(self.lost)
+            if dist.get_backend() == "gloo":
+                for t in (self.sums, self.lost):
+                    h = t.cpu()
+                    dist.all_reduce(h)
+                    t.copy_(h)
+            else:
+                dist.all_reduce(self.sums)
+                dist.all_reduce(self.lost)
 
     def read(self) -> dict:
         """The record after `allreduce`: Eq. 3 on the summed sums, formed by the library."""

@@ -45,6 +45,23 @@ def test_sharded_flow_with_two_emulated_ranks_through_the_benchmarks_own_code():
     assert j["theta_bytes_sent_per_rank_per_step"] == j["params_total"]          # 2 B x half of the parameters x 1 peer
 
 
+def test_sharded_leg_as_two_processes_on_this_gpu():
+    # what `bench.py --gpus N` runs for its "sharded" record, with the two ranks as separate processes on this
+    # one GPU: CUDA IPC handles exchanged, each rank maps the other's theta copy and its step kernel stores
+    # into it; the EDQ sums travel over gloo here (NCCL needs a GPU per rank).  The ranks' kernels never wait
+    # on one another.  Afterwards both processes hold the same full theta.
+    p = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
+                        "--master-addr", "127.0.0.1", "--master-port", "29533", str(ROOT / "bench.py"), "--gpus", "2",
+                        "--sharded-only", "--sharded-backend", "gloo", "--sharded-one-device", "--layers", "0", "--steps", "3",
+                        "--warmup", "2"], cwd=ROOT, capture_output=True, text=True, timeout=900)
+    assert p.returncode == 0, p.stderr[-3000:]
+    j = json.loads([l for l in p.stdout.splitlines() if l.startswith("{")][-1])["sharded_step"]
+    assert "unavailable" not in j, j
+    assert j["ranks"] == 2 and j["copies_agree"] and j["edq_fault"] == 0 and j["edq"] > 0
+    assert j["params_total"] == 262_148_096 and abs(j["params_per_rank"] - j["params_total"] / 2) <= 8
+    assert j["theta_bytes_sent_per_rank_per_step"] == 2 * j["params_per_rank"]
+
+
 @pytest.mark.parametrize("config", [0, 1, 2])
 def test_other_configurations_print_contract_lines(config):
     p = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--config", str(config)], cwd=ROOT, capture_output=True,
