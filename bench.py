@@ -285,6 +285,10 @@ def run_sharded_children(args, world):
            "--sharded-only", "--steps", str(args.steps), "--warmup", str(args.warmup), "--layers", str(args.layers)]
     if args.lib:
         cmd += ["--lib", args.lib]
+    if getattr(args, "sharded_backend", "nccl") != "nccl":
+        cmd += ["--sharded-backend", args.sharded_backend]
+    if getattr(args, "sharded_one_device", False):
+        cmd += ["--sharded-one-device"]
     try:
         proc = subprocess.run(cmd, capture_output=True, text=True, timeout=420, env=env, cwd=str(ROOT))
     except subprocess.TimeoutExpired:

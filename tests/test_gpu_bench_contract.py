@@ -1,5 +1,6 @@
 """bench.py's own arm on a reduced workload: the JSON line carries every key the contract names."""
 import json
+import os
 import subprocess
 import sys
 from pathlib import Path
@@ -50,12 +51,13 @@ def test_sharded_leg_as_two_processes_on_this_gpu():
     # one GPU: CUDA IPC handles exchanged, each rank maps the other's theta copy and its step kernel stores
     # into it; the EDQ sums travel over gloo here (NCCL needs a GPU per rank).  The ranks' kernels never wait
     # on one another.  Afterwards both processes hold the same full theta.
-    p = subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node=2",
-                        "--master-addr", "127.0.0.1", "--master-port", "29533", str(ROOT / "bench.py"), "--gpus", "2",
-                        "--sharded-only", "--sharded-backend", "gloo", "--sharded-one-device", "--layers", "0", "--steps", "3",
-                        "--warmup", "2"], cwd=ROOT, capture_output=True, text=True, timeout=900)
-    assert p.returncode == 0, p.stderr[-3000:]
-    j = json.loads([l for l in p.stdout.splitlines() if l.startswith("{")][-1])["sharded_step"]
+    # launched the way rank 0 of an N-rank run launches it (child processes with their own rendezvous)
+    import argparse
+    sys.path.insert(0, str(ROOT))
+    import bench
+    args = argparse.Namespace(steps=3, warmup=2, layers=0, lib=None, sharded_backend="gloo", sharded_one_device=True)
+    os.environ.setdefault("MASTER_PORT", "29526")
+    j = bench.run_sharded_children(args, 2)
     assert "unavailable" not in j, j
     assert j["ranks"] == 2 and j["copies_agree"] and j["edq_fault"] == 0 and j["edq"] > 0
     assert j["params_total"] == 262_148_096 and abs(j["params_per_rank"] - j["params_total"] / 2) <= 8
