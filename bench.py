@@ -39,8 +39,8 @@ STRATEGY_NAME = {0: "plain_bf16", 1: "collage_light", 2: "collage_plus"}
 STRATEGY = 2                                  # Collage-plus
 WORKLOAD = "llama7b_shaped_291_tensors_collage_plus_with_edq"
 # DRAM bytes per parameter of the step kernel from one ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum = 3.146 GB + 2.565 GB on the 262,148,096-parameter case, summary under
-# profiles/); every byte is touched once, so traffic scales with the parameter count.
+# dram__bytes_write.sum = 3.146 GB + 2.565 GB on the 262,148,096-parameter case: the embedding, final norm
+# and lm_head of the same layout); every byte is touched once, so traffic scales with the parameter count.
 NCU_TRAFFIC_BYTES_PER_PARAM = (3.146280e9 + 2.564761e9) / 262_148_096
 
 
