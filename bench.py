@@ -193,7 +193,7 @@ def run_collage(args):
 
     def step(t):
         if args.per_tensor:
-            B.adamw_step_multi_per_tensor(plan, B.make_hyper(**hyp, edq_out=edq_dev), t, STRATEGY, per, len(rows), cws, stream)
+            B.adamw_step_multi_per_tensor(plan, B.make_hyper(**hyp, flags=pin, edq_out=edq_dev), t, STRATEGY, per, len(rows), cws, stream)
         else:
             B.adamw_step_multi(plan, B.make_hyper(**hyp, flags=pin, edq_out=edq_dev, workspace=ws), t, STRATEGY, stream)
         if use_dist:                                    # EDQ is global: sum the partial sums over ranks

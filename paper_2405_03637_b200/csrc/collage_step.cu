@@ -571,7 +571,10 @@ static cudaError_t dispatch_step2(const StepParams& p, int strategy, bool edq, i
 }
 // multi-tensor step with one EDQ record per chunk
 static cudaError_t dispatch_step_per_chunk(const StepParams& p, int strategy, int sm_count, cudaStream_t stream,
-                                           int* grid_out) {
+                                           int* grid_out, bool large) {
+    if (large && strategy == 2)
+        return p.k.fast ? launch_step<2, true, false, true, true, false, true>(p, sm_count, stream, grid_out)
+                        : launch_step<2, true, false, false, true, false, true>(p, sm_count, stream, grid_out);
     switch (strategy * 2 + (p.k.fast ? 1 : 0)) {
         case 0: return launch_step<0, true, false, false, true>(p, sm_count, stream, grid_out);
         case 1: return launch_step<0, true, false, true, true>(p, sm_count, stream, grid_out);
@@ -1143,7 +1146,9 @@ collage_status_t collage_adamw_step_multi_per_tensor(const collage_plan_t* plan,
         return COLLAGE_ERR_CUDA;
     if (plan->num_chunks > 0) {
         int grid = 0;
-        if (dispatch_step_per_chunk(p, strategy, dev.sm_count, cs, &grid) != cudaSuccess) return COLLAGE_ERR_CUDA;
+        const bool large = plan->chunk_elems % pipe_tile(COLLAGE_PLUS, true) == 0 &&
+                           takes_large_tiles(strategy, p.k.flags, h.flags, plan->num_elements);
+        if (dispatch_step_per_chunk(p, strategy, dev.sm_count, cs, &grid, large) != cudaSuccess) return COLLAGE_ERR_CUDA;
         edq_per_tensor_kernel<<<plan->num_tensors, 256, 0, cs>>>(p.chunk_partials, plan->d_first_chunk, plan->d_orig_index,
                                                                  plan->d_sizes, per_tensor_out_dev);
         if (cudaGetLastError() != cudaSuccess) return COLLAGE_ERR_CUDA;

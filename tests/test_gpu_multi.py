@@ -117,7 +117,7 @@ def test_plan_strategy_needs_its_components():
 
 @pytest.mark.parametrize("strategy", [0, 1, 2])
 @pytest.mark.parametrize("chunk", [0, 2048])
-def test_per_tensor_edq_matches_oracle_tensor_by_tensor(strategy, chunk):
+def test_per_tensor_edq_matches_oracle_tensor_by_tensor(strategy, chunk, step_kernel):
     shapes = W.ragged_shapes() + [("big", 700_001)]
     hyp = W.HYPERS
     host, dev, grads, rows = _build(shapes, strategy, seed=7, misalign_of=lambda i: (0, 1, 0)[i % 3])
