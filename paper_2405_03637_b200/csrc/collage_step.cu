@@ -77,7 +77,16 @@ constexpr PipeGeometry pipe_geometry(int strategy) {
 #ifndef COLLAGE_LARGE_TILE_MIN_N
 #define COLLAGE_LARGE_TILE_MIN_N (1ull << 27)
 #endif
-constexpr PipeGeometry kLargeGeometry = {512, 2, 2};
+#ifndef COLLAGE_LARGE_CONSUMERS
+#define COLLAGE_LARGE_CONSUMERS 512
+#endif
+#ifndef COLLAGE_LARGE_VPT
+#define COLLAGE_LARGE_VPT 2
+#endif
+#ifndef COLLAGE_LARGE_STAGES
+#define COLLAGE_LARGE_STAGES 2
+#endif
+constexpr PipeGeometry kLargeGeometry = {COLLAGE_LARGE_CONSUMERS, COLLAGE_LARGE_VPT, COLLAGE_LARGE_STAGES};
 // elements per tile
 constexpr uint32_t pipe_tile(int strategy, bool large = false) {
     return large ? static_cast<uint32_t>(kLargeGeometry.consumers) * 8u * static_cast<uint32_t>(kLargeGeometry.vpt)
