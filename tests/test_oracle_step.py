@@ -390,3 +390,26 @@ def test_step_lost_count_against_exact_rationals(strategy):
         assert sums["lost"] == want, (strategy, t)
         seen_lost += want
     assert seen_lost > 0
+
+
+def test_edq_sums_against_exactly_rounded_summation():
+    # Eq. 3's two sums as the oracle forms them (double, one pass in index order) against the correctly rounded
+    # sums of the same terms (math.fsum): every term d * eff and d * d is exact in double (8-bit times at most
+    # 17-bit significands), so the only error is the summation's, far below the 1e-5 the device is held to
+    import math
+    n = 1 << 21
+    th = W.bits(W.flat_weights(n, 9)); g = W.bits(W.flat_grads(n, 9, 1))
+    for strategy in (0, 2):
+        st = _state(th.copy(), strategy)
+        sums, d = _step(st, g, 1, strategy, want_delta=True)
+        dd = bits_to_f64(d)
+        eff = bits_to_f64(st["x_hi"]) - bits_to_f64(th)
+        if strategy:
+            eff = eff + bits_to_f64(st["x_lo"])
+        dot, sq = math.fsum((dd * eff).tolist()), math.fsum((dd * dd).tolist())
+        assert sums["dot"] == pytest.approx(dot, rel=1e-12) and sums["sumsq"] == pytest.approx(sq, rel=1e-12)
+        assert sums["edq"] == pytest.approx(dot / math.sqrt(sq), rel=1e-12)
+        # threads only change the association
+        st2 = _state(th.copy(), strategy)
+        sums2, _ = _step(st2, g, 1, strategy, threads=7)
+        assert sums2["dot"] == pytest.approx(dot, rel=1e-12) and sums2["lost"] == sums["lost"]
