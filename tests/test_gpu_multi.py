@@ -49,7 +49,7 @@ def _oracle_multi(host, gbits, t, strategy, hyp):
 
 @pytest.mark.parametrize("strategy", [0, 1, 2])
 @pytest.mark.parametrize("chunk", [0, 2048, 65536])
-def test_ragged_tensor_set(strategy, chunk):
+def test_ragged_tensor_set(strategy, chunk, step_kernel):
     shapes = W.ragged_shapes()
     hyp = W.HYPERS
     host, dev, grads, rows = _build(shapes, strategy, seed=3, misalign_of=lambda i: (0, 0, 1, 0, 0, 3)[i % 6])
@@ -162,7 +162,7 @@ def test_per_tensor_edq_matches_oracle_tensor_by_tensor(strategy, chunk, step_ke
 
 
 @pytest.mark.parametrize("strategy", [0, 2])
-def test_theta_replicas_are_written_by_the_step_itself(strategy):
+def test_theta_replicas_are_written_by_the_step_itself(strategy, step_kernel):
     # sharded optimizer state needs theta everywhere: the step writes it to registered replicas (here two more
     # buffers on this GPU; on several GPUs they would be peers' memory) - ragged, unaligned and empty tensors included
     shapes = W.ragged_shapes() + [("big", 500_003)]
@@ -205,7 +205,7 @@ def test_theta_replicas_are_written_by_the_step_itself(strategy):
 
 
 @pytest.mark.parametrize("world", [2, 3])
-def test_sharded_step_of_emulated_ranks_gathers_theta_everywhere(world):
+def test_sharded_step_of_emulated_ranks_gathers_theta_everywhere(world, step_kernel):
     # ZeRO-1-style ownership on one device: every "rank" keeps its own full copy of theta (what its forward
     # pass would read) and the optimizer state of its slice only; its step writes the new theta of the slice
     # into every rank's copy.  The ranks' kernels do not wait on one another, so running them one after the
